@@ -1,0 +1,249 @@
+/*
+ * isv.h - decode attention over a paged KV cache that is split between GPU HBM
+ * and pinned host memory (KV cache offloading), for NVIDIA B200 (sm_100a).
+ *
+ * The library executes the computation whose time the InferSave cost model
+ * predicts per layer and decode step (paper Section IV-C, Eq. 6):
+ *     T_dec = CTCF(T_compute^d) + T_trans^d
+ * i.e. the self-attention part of T_compute^d (4 * BS * ctx * h1 flops) over a
+ * KV cache of which the fraction C_off (Section IV-B) lives in CPU memory and
+ * must cross the host link (T_trans^d) every step.
+ *
+ * Conventions
+ *   - All entry points return 0 (ISV_OK) or a negative ISV_E* code; the text of
+ *     the last error of the calling thread is available from isv_last_error().
+ *     Nothing aborts, throws across the boundary or traps on the device.
+ *   - "device" pointers are CUDA device addresses on the GPU that was current
+ *     when the handle was created; "host" pointers are ordinary CPU addresses.
+ *   - Work is enqueued on the handle's compute stream (and on internal copy
+ *     streams) and is asynchronous unless a function says it synchronises.
+ *     Caller-owned buffers must stay valid until that work has completed.
+ *   - K/V/q/out elements are 16-bit (fp16 or bf16, chosen at allocation);
+ *     arithmetic is fp32.
+ *   - KV pool layout, per physical layer and pool (HBM pool, host pool):
+ *         [block][K|V][kv_head][block_tokens][head_dim]
+ *     so one (block, K-or-V, head) tile is contiguous.
+ *   - Block table entry (int32): ISV_BLOCK_NONE = not allocated; otherwise the
+ *     physical block id, with ISV_BLOCK_HOST_BIT set when the block belongs to
+ *     the host pool.  The block that holds a sequence's newest token is kept in
+ *     GPU memory even when it is host-flagged (it is still being written); it
+ *     is copied to the host pool when it becomes full.
+ */
+#ifndef ISV_H
+#define ISV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ISV_OK               0
+#define ISV_EINVAL          (-1)   /* bad argument                                   */
+#define ISV_ENOMEM_DEVICE   (-2)   /* cudaMalloc refused                             */
+#define ISV_ENOMEM_PINNED   (-3)   /* pinned host allocation refused                 */
+#define ISV_ECAPACITY       (-4)   /* sequence or pool would exceed its capacity     */
+#define ISV_ECUDA           (-5)   /* a CUDA runtime call failed                     */
+#define ISV_ETIMEOUT        (-6)   /* a bounded wait ran out                         */
+#define ISV_EDEVICE_STATUS  (-7)   /* a kernel reported a problem (see status bits)  */
+#define ISV_ENODEVICE       (-8)   /* compute requested on a plan-only handle        */
+
+#define ISV_F16   0
+#define ISV_BF16  1
+
+#define ISV_BLOCK_NONE      (-1)
+#define ISV_BLOCK_HOST_BIT  (1 << 30)
+
+/* bits of the device status word (isv_step_times.status, isv_device_status) */
+#define ISV_STATUS_BAD_BLOCK_ID  1u   /* a table entry pointed outside its pool; block skipped */
+#define ISV_STATUS_WAIT_EXPIRED  2u   /* a bounded wait inside a kernel gave up                */
+
+typedef struct isv_kv isv_kv;   /* opaque; created by isv_kv_alloc, destroyed by isv_kv_free */
+
+/*
+ * Problem statement of one cache (paper Table II: model shape, batch size,
+ * input/output lengths, precision; Section IV-B: offload ratio).
+ */
+typedef struct {
+    int32_t  layers;             /* logical layers (n)                                          */
+    int32_t  phys_layers;        /* physical KV slabs; 0 = layers.  Logical layer l uses slab   */
+                                 /* l % phys_layers (lets a benchmark hold fewer slabs than     */
+                                 /* layers; layers sharing a slab overwrite each other's data)  */
+    int32_t  q_heads;            /* query heads; multiple of kv_heads                           */
+    int32_t  kv_heads;
+    int32_t  head_dim;           /* 64 or 128                                                   */
+    int32_t  block_tokens;       /* tokens per KV block; 16                                     */
+    int32_t  dtype;              /* ISV_F16 or ISV_BF16                                         */
+    float    offload_frac;       /* C_off in [0, 1]: of every prefix of j blocks of a sequence, */
+                                 /* floor(j * C_off) are host-resident                          */
+    int32_t  max_seqs;           /* capacity in sequences (BS), <= 4096                         */
+    int32_t  max_tokens_per_seq; /* capacity per sequence (L_in + L_out)                        */
+    uint64_t perm_seed;          /* 0 = physical block ids handed out in order; otherwise they  */
+                                 /* follow a seeded permutation (host pool ids stay compact)    */
+    uint64_t chunk_bytes;        /* staging chunk size; 0 = 32 MiB                              */
+    int32_t  ring_depth;         /* staging ring buffers; 0 = 3                                 */
+    int32_t  split_blocks;       /* KV blocks per split of the resident kernel; 0 = 8           */
+    int32_t  plan_only;          /* 1 = host bookkeeping only: no CUDA call is made, no memory  */
+                                 /* is allocated, compute entry points return ISV_ENODEVICE     */
+    void    *compute_stream;     /* cudaStream_t to enqueue on, or NULL = library creates one   */
+                                 /* (the legacy default stream, handle 0, cannot be passed)     */
+} isv_kv_desc;
+
+/* Sizes the library derived from a description (filled by isv_kv_info). */
+typedef struct {
+    uint64_t block_bytes;        /* one block: 2 * kv_heads * block_tokens * head_dim * 2 B     */
+    uint64_t kv_bytes_per_token; /* K and V of one token in one layer                           */
+    int32_t  max_blocks_per_seq;
+    int32_t  hbm_blocks;         /* HBM pool capacity per physical layer, in blocks             */
+    int32_t  host_blocks;        /* host pool capacity per physical layer, in blocks            */
+    int32_t  hbm_blocks_used;
+    int32_t  host_blocks_used;
+    uint64_t hbm_pool_bytes;     /* all physical layers, tail slots included                    */
+    uint64_t host_pool_bytes;    /* all physical layers                                         */
+    uint64_t scratch_bytes;      /* partials, running state, staging ring                       */
+    int32_t  phys_layers;
+    int32_t  split_blocks;
+    int32_t  ring_depth;
+    int32_t  sm_count;
+    uint64_t chunk_bytes;
+    uint64_t kernel_launches;    /* kernels this handle has launched since it was created       */
+} isv_kv_info_t;
+
+/*
+ * Per-layer timing of the most recent decode of that layer, and what the
+ * paper's terms are for it: h2d_ms is T_trans^d, attn_resident_ms +
+ * attn_offloaded_ms + merge_ms is the self-attention part of T_compute^d,
+ * total_ms is T_dec without the linear layers.  Byte counters: bytes_resident
+ * and bytes_offloaded are the KV bytes the attention had to read from HBM and
+ * to fetch over the host link; bytes_offloaded equals the first term of the
+ * T_trans^d numerator, C_off * 2 * L * h1 * Precision * BS, counted per block.
+ * bytes_staged is what the copy engine actually moved (whole chunks).
+ */
+typedef struct {
+    float    append_ms;
+    float    h2d_ms;
+    float    attn_resident_ms;
+    float    attn_offloaded_ms;
+    float    merge_ms;
+    float    total_ms;
+    uint64_t bytes_resident;
+    uint64_t bytes_offloaded;
+    uint64_t bytes_staged;
+    uint64_t bytes_appended;
+    int32_t  n_chunks;
+    uint32_t status;
+} isv_step_times;
+
+/* ---- lifetime ---------------------------------------------------------- */
+
+/* Allocates pools (HBM, pinned host), block tables, scratch, staging ring,
+ * streams and events on the current device.  Synchronous.  *out is NULL on
+ * failure.  The handle must be used from one host thread at a time. */
+int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc);
+
+/* Waits for all work of the handle, then frees everything it owns. */
+int isv_kv_free(isv_kv *h);
+
+/* Forgets all sequences (lengths 0, all blocks free).  Synchronises. */
+int isv_kv_reset(isv_kv *h);
+
+int isv_kv_info(isv_kv *h, isv_kv_info_t *out);
+
+/* ---- loading and appending (the KV cache of Section II-A) --------------- */
+
+/* Prompt load for one layer (prefill's KV, not timed): k, v are device arrays
+ * [n_seqs][T][kv_heads][head_dim]; lens_host[s] <= T tokens of sequence s are
+ * kept and replace what the layer held for s.  Blocks are allocated by the
+ * residency rule on first use and shared by all layers.  Synchronises. */
+int isv_kv_fill(isv_kv *h, int32_t layer, const void *k_dev, const void *v_dev,
+                const int32_t *lens_host, int32_t n_seqs, int32_t T);
+
+/* Appends one token to sequences 0..n_seqs-1 of one layer at that layer's
+ * current lengths (the cache growth of one decode step): k, v are device
+ * arrays [n_seqs][kv_heads][head_dim].  K and V are written by one kernel; the
+ * copy is bit-exact.  ISV_ECAPACITY if a sequence is full. */
+int isv_kv_append(isv_kv *h, int32_t layer, const void *k_dev, const void *v_dev,
+                  int32_t n_seqs);
+
+/* ---- decode attention (self-attention term of T_compute^d; T_trans^d) ---- */
+
+/* out[s][h][:] = softmax(q[s][h] . K_s^T / sqrt(head_dim)) V_s over the
+ * layer's current tokens of sequence s (the newest token included), for
+ * s < n_seqs.  q_dev: [n_seqs][q_heads][head_dim] 16-bit; out_dev (same shape
+ * and dtype) and out_f32_dev (fp32) may each be NULL but not both.  Query head
+ * h reads KV head h / (q_heads / kv_heads).  A sequence of length 0 yields
+ * zeros.  Host-resident blocks are streamed through the staging ring on the
+ * copy stream while the resident blocks are processed; partial results are
+ * combined by a log-sum-exp merge.
+ * block_table_dev / seq_lens_dev: NULL = the library's own (normal use).  If
+ * given, they replace the library's device arrays for the resident kernel
+ * (same format, row stride as isv_block_table_dev reports) and must agree with
+ * the library's bookkeeping on lengths and on host-resident entries. */
+int isv_attn_decode(isv_kv *h, int32_t layer, const void *q_dev, void *out_dev,
+                    float *out_f32_dev, const int32_t *block_table_dev,
+                    const int32_t *seq_lens_dev, int32_t n_seqs);
+
+/* One decode step of all layers: for l in 0..layers-1 append then attend.
+ * Device arrays: q, out [layers][n_seqs][q_heads][head_dim];
+ * k, v [layers][n_seqs][kv_heads][head_dim]. */
+int isv_decode_step(isv_kv *h, const void *q_dev, const void *k_dev, const void *v_dev,
+                    void *out_dev, int32_t n_seqs);
+
+/* The same step with HOST buffers of the same shapes (pinned memory gives
+ * asynchronous copies): inputs are copied to library-owned device buffers,
+ * the step runs, out is copied back.  Returns after the result is in
+ * out_host (synchronises). */
+int isv_decode_step_host(isv_kv *h, const void *q_host, const void *k_host,
+                         const void *v_host, void *out_host, int32_t n_seqs);
+
+/* ---- inspection --------------------------------------------------------- */
+
+/* Logical-order copy of one sequence's K and V of one layer to host arrays
+ * [len][kv_heads][head_dim] (capacity max_tokens_per_seq rows each).
+ * Bit-exact; synchronises. */
+int isv_kv_gather(isv_kv *h, int32_t layer, int32_t seq, void *k_host, void *v_host,
+                  int32_t *len_out);
+
+/* Library-maintained device arrays: table [max_seqs][*row_stride] int32 and
+ * one layer's lengths [max_seqs] int32.  NULL on a plan-only handle. */
+const int32_t *isv_block_table_dev(isv_kv *h, int32_t *row_stride);
+const int32_t *isv_seq_lens_dev(isv_kv *h, int32_t layer);
+
+/* Host copies of the same (work on plan-only handles too). */
+int isv_block_table_host(isv_kv *h, int32_t *out, int32_t n_seqs, int32_t row_stride);
+int isv_seq_lens_host(isv_kv *h, int32_t layer, int32_t *out, int32_t n_seqs);
+
+/* KV bytes a decode of this layer over n_seqs sequences would read now:
+ * resident (HBM) and offloaded (host link) algorithmic bytes, the bytes the
+ * staging engine would copy, and its chunk count.  Any pointer may be NULL. */
+int isv_plan_bytes(isv_kv *h, int32_t layer, int32_t n_seqs, uint64_t *bytes_resident,
+                   uint64_t *bytes_offloaded, uint64_t *bytes_staged, int32_t *n_chunks);
+
+/* ---- timing (feeds the terms of Eq. 6) ----------------------------------- */
+
+/* Turns event recording per layer on or off (off by default: events cost a
+ * little on short steps). */
+int isv_set_timing(isv_kv *h, int32_t on);
+
+/* Times of the latest decode of `layer`, or with layer = -1 the sums over all
+ * layers (total_ms then spans first layer start to last layer end).
+ * Synchronises.  Times are 0 where timing was off. */
+int isv_step_timing(isv_kv *h, int32_t layer, isv_step_times *out);
+
+/* Waits for everything enqueued by the handle; returns ISV_EDEVICE_STATUS if
+ * a kernel flagged a problem since the last call (bits in *status_out). */
+int isv_sync(isv_kv *h, uint32_t *status_out);
+
+/* Measures pinned host<->device copy bandwidth on the current device: `bytes`
+ * per copy, best of `reps`, CUDA events.  This is the measured host-link rate
+ * that T_trans^d's BW_cpu->gpu stands for.  Allocates and frees its buffers. */
+int isv_link_probe(uint64_t bytes, int32_t reps, double *h2d_gbs, double *d2h_gbs);
+
+/* Text of the calling thread's last error; valid until its next call. */
+const char *isv_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ISV_H */

@@ -1,0 +1,824 @@
+// CUDA kernels of the offloaded-KV decode path (sm_100a):
+//   decode_kernel   split flash-decoding over paged K/V tiles, persistent CTAs,
+//                   one autonomous TMA-fed pipeline per warp
+//   merge_kernel    log-sum-exp merge of the resident result and the
+//                   offloaded running state
+//   append_kernel   K and V of one new token per sequence, one launch
+//   fill / gather   prompt load and logical-order read-back
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/isv.h"
+#include "isv_kernels.cuh"
+
+namespace isv {
+
+namespace {
+
+constexpr float kNegBig = -1.0e30f;          // "no score yet": finite so differences never give NaN
+constexpr uint32_t kFull = 0xffffffffu;
+constexpr uint32_t kSpinLimit = 1u << 22;    // polls before a wait gives up
+
+// ---------------------------------------------------------------- PTX helpers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the phase did not complete within kSpinLimit polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 256) __nanosleep(64);
+    }
+    return false;
+}
+// 1-D bulk copy global -> shared of this CTA, completion counted on an mbarrier.
+// Addresses and size are multiples of 16 bytes by construction of the pool layout.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+
+template <bool BF16>
+__device__ __forceinline__ void cvt8(const uint4 &r, float (&f)[8]) {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (BF16) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        } else {
+            const __half2 h = *reinterpret_cast<const __half2 *>(&w[i]);
+            const float2 t = __half22float2(h);
+            f[2 * i] = t.x;
+            f[2 * i + 1] = t.y;
+        }
+    }
+}
+
+template <bool BF16>
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+    if (BF16) {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+        return *reinterpret_cast<const uint32_t *>(&h);
+    } else {
+        const __half2 h = __floats2half2_rn(a, b);
+        return *reinterpret_cast<const uint32_t *>(&h);
+    }
+}
+
+// ---------------------------------------------------------------- one K/V tile
+
+// Lane layout inside a warp: grp = lane / 8 owns tokens grp, grp+4, ... of the
+// tile; sub = lane % 8 owns head-dim elements [v*64 + sub*8, +8) for v < D/64.
+// Each group keeps its own running (m, l, o); groups are merged at unit end.
+template <int D, int GT, int BT, bool BF16>
+__device__ __forceinline__ void tile_compute(const uint8_t *sK, const uint8_t *sV, int ntok, int grp, int sub,
+                                             const float (&q)[GT][D / 8], float (&o)[GT][D / 8], float (&m)[GT],
+                                             float (&l)[GT]) {
+    constexpr int NV = D / 64, NQ = BT / 4, ROW = D * 2;
+    float sc[NQ][GT];
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) {
+        const int t = 4 * i + grp;
+        const uint4 *kp = reinterpret_cast<const uint4 *>(sK + t * ROW) + sub;
+        float acc[GT];
+#pragma unroll
+        for (int g = 0; g < GT; ++g) acc[g] = 0.f;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            float kf[8];
+            cvt8<BF16>(kp[v * 8], kf);
+#pragma unroll
+            for (int g = 0; g < GT; ++g)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g] = fmaf(q[g][v * 8 + e], kf[e], acc[g]);
+        }
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            float a = acc[g];
+            a += __shfl_xor_sync(kFull, a, 4);
+            a += __shfl_xor_sync(kFull, a, 2);
+            a += __shfl_xor_sync(kFull, a, 1);
+            sc[i][g] = (t < ntok) ? a : kNegBig;
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < GT; ++g) {
+        float mx = sc[0][g];
+#pragma unroll
+        for (int i = 1; i < NQ; ++i) mx = fmaxf(mx, sc[i][g]);
+        if (mx > m[g]) {
+            const float r = exp2f(m[g] - mx);
+            l[g] *= r;
+#pragma unroll
+            for (int e = 0; e < D / 8; ++e) o[g][e] *= r;
+            m[g] = mx;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) {
+        const int t = 4 * i + grp;
+        if (t < ntok) {   // slots past the sequence end hold unspecified bits: never touch them
+            float pw[GT];
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                pw[g] = exp2f(sc[i][g] - m[g]);
+                l[g] += pw[g];
+            }
+            const uint4 *vp = reinterpret_cast<const uint4 *>(sV + t * ROW) + sub;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                float vf[8];
+                cvt8<BF16>(vp[v * 8], vf);
+#pragma unroll
+                for (int g = 0; g < GT; ++g)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) o[g][v * 8 + e] = fmaf(pw[g], vf[e], o[g][v * 8 + e]);
+            }
+        }
+    }
+}
+
+// Stores one row held in group layout (lanes 0..7 cover the row).
+template <int D, bool BF16>
+__device__ __forceinline__ void store_row_grouped(void *out, float *out_f32, size_t row, int sub,
+                                                  const float (&o)[D / 8], float scale) {
+#pragma unroll
+    for (int v = 0; v < D / 64; ++v) {
+        float x[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] = o[v * 8 + e] * scale;
+        const size_t idx = row * D + v * 64 + sub * 8;
+        if (out_f32) {
+            *reinterpret_cast<float4 *>(out_f32 + idx) = make_float4(x[0], x[1], x[2], x[3]);
+            *reinterpret_cast<float4 *>(out_f32 + idx + 4) = make_float4(x[4], x[5], x[6], x[7]);
+        }
+        if (out) {
+            uint4 w;
+            w.x = pack2<BF16>(x[0], x[1]);
+            w.y = pack2<BF16>(x[2], x[3]);
+            w.z = pack2<BF16>(x[4], x[5]);
+            w.w = pack2<BF16>(x[6], x[7]);
+            *reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(out) + idx) = w;
+        }
+    }
+}
+
+// Last-arriving unit of a (sequence, head group): combine the nu partials of
+// query head g.  Lane owns D/32 consecutive elements.
+template <int D, bool BF16>
+__device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int u0, int nu, int g, int GT,
+                                                   size_t row, int lane) {
+    constexpr int EPL = D / 32;
+    float mm = kNegBig;
+    for (int c = lane; c < nu; c += 32) mm = fmaxf(mm, __ldcg(&p.part_ml[((size_t)(u0 + c) * GT + g) * 2]));
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) mm = fmaxf(mm, __shfl_xor_sync(kFull, mm, d));
+    float ll = 0.f;
+    float acc[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+    for (int c = 0; c < nu; ++c) {
+        const size_t pr = (size_t)(u0 + c) * GT + g;
+        const float2 ml = __ldcg(reinterpret_cast<const float2 *>(&p.part_ml[pr * 2]));
+        const float a = exp2f(ml.x - mm);
+        ll += ml.y * a;
+        const float *po = p.part_o + pr * D + lane * EPL;
+        if (EPL == 4) {
+            const float4 x = __ldcg(reinterpret_cast<const float4 *>(po));
+            acc[0] = fmaf(a, x.x, acc[0]);
+            acc[1] = fmaf(a, x.y, acc[1]);
+            acc[2] = fmaf(a, x.z, acc[2]);
+            acc[3] = fmaf(a, x.w, acc[3]);
+        } else {
+            const float2 x = __ldcg(reinterpret_cast<const float2 *>(po));
+            acc[0] = fmaf(a, x.x, acc[0]);
+            acc[1] = fmaf(a, x.y, acc[1]);
+        }
+    }
+    const size_t idx = row * D + lane * EPL;
+    if (p.finalize) {
+        const float inv = ll > 0.f ? 1.f / ll : 0.f;
+        if (p.out_f32) {
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) p.out_f32[idx + e] = acc[e] * inv;
+        }
+        if (p.out) {
+            uint16_t *o16 = reinterpret_cast<uint16_t *>(p.out) + idx;
+            if (EPL == 4) {
+                uint2 w;
+                w.x = pack2<BF16>(acc[0] * inv, acc[1] * inv);
+                w.y = pack2<BF16>(acc[2] * inv, acc[3] * inv);
+                *reinterpret_cast<uint2 *>(o16) = w;
+            } else {
+                *reinterpret_cast<uint32_t *>(o16) = pack2<BF16>(acc[0] * inv, acc[1] * inv);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) p.acc_o[idx + e] = acc[e];
+        if (lane == 0) {
+            p.acc_ml[row * 2] = mm;
+            p.acc_ml[row * 2 + 1] = ll;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- decode kernel
+
+// Stage metadata words written by the producing lane before it arms the stage.
+enum { M_UNIT = 0, M_SEQ, M_HG, M_C, M_NU, M_NTOK, M_LAST, M_WORDS = 8 };
+
+template <int D, int GT, int BT, bool BF16, int MODE>
+__global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const DecodeParams p, const int stages) {
+    constexpr uint32_t TILE = BT * D * 2;
+    constexpr uint32_t STAGE = 2 * TILE;
+    constexpr int E = D / 8;
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int grp = lane >> 3, sub = lane & 7;
+
+    uint8_t *data = smem + (size_t)warp * stages * STAGE;
+    uint8_t *after_data = smem + (size_t)kDecodeWarps * stages * STAGE;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(after_data) + warp * stages;
+    int32_t *meta = reinterpret_cast<int32_t *>(after_data + (size_t)kDecodeWarps * stages * 8) +
+                    warp * stages * M_WORDS;
+    int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)kDecodeWarps * stages * (8 + 4 * M_WORDS));
+
+    const int Hg = p.Hkv * p.P;
+    const uint64_t block_bytes = p.block_bytes;
+
+    // ---- unit count and this warp's contiguous range of units
+    int NU;
+    if (MODE == MODE_RESIDENT) {
+        for (int s = threadIdx.x; s < p.n_seqs; s += blockDim.x) {
+            const int len = p.lens[s];
+            const int nblk = (len + BT - 1) / BT;
+            const int nu = max(1, (nblk + p.U - 1) / p.U);
+            ubase[s + 1] = nu * Hg;
+        }
+        if (threadIdx.x == 0) ubase[0] = 0;
+        __syncthreads();
+        if (warp == 0) {
+            int carry = 0;
+            for (int base = 0; base < p.n_seqs; base += 32) {
+                const int i = base + lane;
+                int v = i < p.n_seqs ? ubase[i + 1] : 0;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int t = __shfl_up_sync(kFull, v, d);
+                    if (lane >= d) v += t;
+                }
+                if (i < p.n_seqs) ubase[i + 1] = carry + v;
+                carry += __shfl_sync(kFull, v, 31);
+            }
+        }
+        __syncthreads();
+        NU = ubase[p.n_seqs];
+    } else {
+        NU = p.cu_count * Hg;
+    }
+    const long long nwt = (long long)gridDim.x * kDecodeWarps;
+    const long long gw = (long long)blockIdx.x * kDecodeWarps + warp;
+    int u_next = (int)((long long)NU * gw / nwt);
+    const int u_end = (int)((long long)NU * (gw + 1) / nwt);
+    if (u_next >= u_end) return;
+
+    if (lane == 0) {
+        for (int st = 0; st < stages; ++st) mbar_init(smem_u32(&bars[st]), 1);
+        fence_barrier_init();
+    }
+    __syncwarp();
+
+    // ---- producer state (identical in all lanes except `ent`)
+    int pu_unit = -1, pu_s = 0, pu_hg = 0, pu_c = 0, pu_nu = 1;
+    int pu_len = 0, pu_jlast = -1, pu_j0 = 0, pu_n = 0;   // entries of the open unit: [pu_j0, pu_j0 + pu_n)
+    int pu_batch = 0, pu_nbatch = 0, pu_base = 0;
+    uint32_t pu_mask = 0;
+    int32_t ent = ISV_BLOCK_NONE;
+    bool pu_open = false, pu_done = false;
+    int prod_stage = 0, inflight = 0;
+    if (MODE == MODE_RESIDENT) {   // sequence of the first unit: largest s with ubase[s] <= u_next
+        int lo = 0, hi = p.n_seqs - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (ubase[mid] <= u_next) lo = mid; else hi = mid - 1;
+        }
+        pu_s = lo;
+    }
+
+    // Emits at most one stage (a tile, or an end-of-unit marker without data).
+    auto produce = [&]() {
+        while (true) {
+            if (pu_mask != 0) {
+                const int i = __ffs(pu_mask) - 1;
+                pu_mask &= pu_mask - 1;
+                const int32_t e = __shfl_sync(kFull, ent, i);
+                const bool last = (pu_mask == 0) && (pu_batch >= pu_nbatch);
+                int ntok = BT;
+                const uint8_t *src;
+                if (MODE == MODE_RESIDENT) {
+                    const int j = pu_base + i;
+                    if (j == pu_jlast) ntok = pu_len - j * BT;
+                    src = (e & ISV_BLOCK_HOST_BIT) ? p.tail + (uint64_t)pu_s * block_bytes
+                                                   : p.pool + (uint64_t)e * block_bytes;
+                } else {
+                    src = p.pool + (uint64_t)e * block_bytes;
+                }
+                const int kvh = pu_hg / p.P;
+                if (lane == 0) {
+                    int32_t *mt = meta + prod_stage * M_WORDS;
+                    mt[M_UNIT] = pu_unit; mt[M_SEQ] = pu_s; mt[M_HG] = pu_hg; mt[M_C] = pu_c;
+                    mt[M_NU] = pu_nu; mt[M_NTOK] = ntok; mt[M_LAST] = last ? 1 : 0;
+                    const uint32_t bar = smem_u32(&bars[prod_stage]);
+                    const uint32_t dst = smem_u32(data + (size_t)prod_stage * STAGE);
+                    mbar_arrive_expect_tx(bar, STAGE);
+                    bulk_g2s(dst, src + (uint64_t)kvh * TILE, TILE, bar);
+                    bulk_g2s(dst + TILE, src + (uint64_t)(p.Hkv + kvh) * TILE, TILE, bar);
+                }
+                if (last) pu_open = false;
+                prod_stage = (prod_stage + 1 == stages) ? 0 : prod_stage + 1;
+                ++inflight;
+                return;
+            }
+            if (pu_open) {
+                if (pu_batch < pu_nbatch) {   // next 32 entries of the unit
+                    pu_base = pu_j0 + 32 * pu_batch;
+                    ++pu_batch;
+                    const int j = pu_base + lane;
+                    bool valid = false;
+                    int32_t e = ISV_BLOCK_NONE;
+                    if (j < pu_j0 + pu_n) {
+                        if (MODE == MODE_RESIDENT) {
+                            e = p.table[(size_t)pu_s * p.table_stride + j];
+                            if (e != ISV_BLOCK_NONE) {
+                                if (e & ISV_BLOCK_HOST_BIT) {
+                                    valid = (j == pu_jlast) && (p.tail != nullptr);
+                                } else {
+                                    valid = e >= 0 && e < p.n_pool_blocks;
+                                    if (!valid) atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+                                }
+                            }
+                        } else {
+                            e = p.cblk[j];
+                            valid = e >= 0 && e < p.n_pool_blocks;
+                            if (!valid) atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+                        }
+                    }
+                    ent = e;
+                    pu_mask = __ballot_sync(kFull, valid);
+                    continue;
+                }
+                // no tile carried the end flag (or the unit is empty): explicit end marker
+                if (lane == 0) {
+                    int32_t *mt = meta + prod_stage * M_WORDS;
+                    mt[M_UNIT] = pu_unit; mt[M_SEQ] = pu_s; mt[M_HG] = pu_hg; mt[M_C] = pu_c;
+                    mt[M_NU] = pu_nu; mt[M_NTOK] = 0; mt[M_LAST] = 1;
+                    mbar_arrive(smem_u32(&bars[prod_stage]));
+                }
+                pu_open = false;
+                prod_stage = (prod_stage + 1 == stages) ? 0 : prod_stage + 1;
+                ++inflight;
+                return;
+            }
+            if (u_next >= u_end) { pu_done = true; return; }
+            // open the next unit
+            pu_unit = u_next++;
+            if (MODE == MODE_RESIDENT) {
+                while (pu_unit >= ubase[pu_s + 1]) ++pu_s;
+                pu_len = p.lens[pu_s];
+                const int nblk = (pu_len + BT - 1) / BT;
+                pu_nu = max(1, (nblk + p.U - 1) / p.U);
+                const int r = pu_unit - ubase[pu_s];
+                pu_hg = r / pu_nu;
+                pu_c = r - pu_hg * pu_nu;
+                pu_j0 = pu_c * p.U;
+                pu_n = max(0, min(p.U, nblk - pu_j0));
+                pu_jlast = nblk - 1;
+            } else {
+                const int cu = p.cu_first + pu_unit / Hg;
+                pu_hg = pu_unit % Hg;
+                pu_s = p.cu_seq[cu];
+                pu_j0 = p.cu_beg[cu];
+                pu_n = p.cu_end[cu] - pu_j0;
+                pu_c = 0;
+                pu_nu = 1;
+            }
+            pu_nbatch = (pu_n + 31) >> 5;
+            pu_batch = 0;
+            pu_mask = 0;
+            pu_open = true;
+        }
+    };
+
+    for (int i = 0; i < stages && !pu_done; ++i) produce();
+
+    // ---- consumer
+    float q[GT][E], o[GT][E], m[GT], l[GT];
+    int cur_unit = -1;
+    int cons_stage = 0;
+    uint32_t cons_phase = 0;
+    while (inflight > 0) {
+        const bool ok = mbar_wait(smem_u32(&bars[cons_stage]), cons_phase);
+        if (!__all_sync(kFull, ok)) {
+            if (lane == 0) atomicOr(p.status, ISV_STATUS_WAIT_EXPIRED);
+            // give copies that may still be in flight one more bounded chance to land, then leave
+            for (int k = 0; k < inflight; ++k) {
+                mbar_wait(smem_u32(&bars[cons_stage]), cons_phase);
+                cons_stage = (cons_stage + 1 == stages) ? 0 : cons_stage + 1;
+                if (cons_stage == 0) cons_phase ^= 1u;
+            }
+            return;
+        }
+        const int32_t *mt = meta + cons_stage * M_WORDS;
+        const int unit = mt[M_UNIT], s = mt[M_SEQ], hg = mt[M_HG], c = mt[M_C], nu = mt[M_NU];
+        const int ntok = mt[M_NTOK];
+        const bool last = mt[M_LAST] != 0;
+        if (unit != cur_unit) {
+            cur_unit = unit;
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                const uint16_t *qrow =
+                    reinterpret_cast<const uint16_t *>(p.q) + ((size_t)s * p.Hq + (size_t)hg * GT + g) * D;
+#pragma unroll
+                for (int v = 0; v < D / 64; ++v) {
+                    const uint4 r = __ldg(reinterpret_cast<const uint4 *>(qrow + v * 64 + sub * 8));
+                    float qf[8];
+                    cvt8<BF16>(r, qf);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) q[g][v * 8 + e] = qf[e] * p.scale_log2;
+                }
+                m[g] = kNegBig;
+                l[g] = 0.f;
+#pragma unroll
+                for (int e = 0; e < E; ++e) o[g][e] = 0.f;
+            }
+        }
+        if (ntok > 0) {
+            const uint8_t *sK = data + (size_t)cons_stage * STAGE;
+            tile_compute<D, GT, BT, BF16>(sK, sK + TILE, ntok, grp, sub, q, o, m, l);
+        }
+        __syncwarp();   // every lane is done with this stage (data and metadata) before it is refilled
+        --inflight;
+        cons_stage = (cons_stage + 1 == stages) ? 0 : cons_stage + 1;
+        if (cons_stage == 0) cons_phase ^= 1u;
+        if (!pu_done) produce();
+
+        if (!last) continue;
+
+        // ---- end of unit: merge the four token groups of the warp
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            float mm = fmaxf(m[g], __shfl_xor_sync(kFull, m[g], 8));
+            mm = fmaxf(mm, __shfl_xor_sync(kFull, mm, 16));
+            const float r = exp2f(m[g] - mm);
+            float ll = l[g] * r;
+            ll += __shfl_xor_sync(kFull, ll, 8);
+            ll += __shfl_xor_sync(kFull, ll, 16);
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                float x = o[g][e] * r;
+                x += __shfl_xor_sync(kFull, x, 8);
+                x += __shfl_xor_sync(kFull, x, 16);
+                o[g][e] = x;
+            }
+            m[g] = mm;
+            l[g] = ll;
+        }
+
+        if (MODE == MODE_STAGED) {
+            // fold into the running state of (s, head); this unit is its only writer in this launch
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                const size_t row = (size_t)s * p.Hq + (size_t)hg * GT + g;
+                const float2 ml = *reinterpret_cast<const float2 *>(&p.acc_ml[row * 2]);
+                if (ml.y > 0.f) {
+                    const float mm = fmaxf(m[g], ml.x);
+                    const float a1 = exp2f(m[g] - mm), a2 = exp2f(ml.x - mm);
+                    l[g] = l[g] * a1 + ml.y * a2;
+#pragma unroll
+                    for (int v = 0; v < D / 64; ++v)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            o[g][v * 8 + e] =
+                                o[g][v * 8 + e] * a1 + p.acc_o[row * D + v * 64 + sub * 8 + e] * a2;
+                    m[g] = mm;
+                }
+                __syncwarp();   // all lanes have read the old state before group 0 overwrites it
+                if (grp == 0) {
+                    store_row_grouped<D, BF16>(nullptr, p.acc_o, row, sub, o[g], 1.f);
+                    if (sub == 0) {
+                        p.acc_ml[row * 2] = m[g];
+                        p.acc_ml[row * 2 + 1] = l[g];
+                    }
+                }
+            }
+            continue;
+        }
+
+        // ---- resident mode
+        if (nu == 1) {   // the unit covered the whole sequence: no partial needed
+            if (grp == 0) {
+#pragma unroll
+                for (int g = 0; g < GT; ++g) {
+                    const size_t row = (size_t)s * p.Hq + (size_t)hg * GT + g;
+                    if (p.finalize) {
+                        store_row_grouped<D, BF16>(p.out, p.out_f32, row, sub, o[g], l[g] > 0.f ? 1.f / l[g] : 0.f);
+                    } else {
+                        store_row_grouped<D, BF16>(nullptr, p.acc_o, row, sub, o[g], 1.f);
+                        if (sub == 0) {
+                            p.acc_ml[row * 2] = m[g];
+                            p.acc_ml[row * 2 + 1] = l[g];
+                        }
+                    }
+                }
+            }
+            continue;
+        }
+        if (grp == 0) {
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                const size_t pr = (size_t)unit * GT + g;
+                store_row_grouped<D, BF16>(nullptr, p.part_o, pr, sub, o[g], 1.f);
+                if (sub == 0) {
+                    p.part_ml[pr * 2] = m[g];
+                    p.part_ml[pr * 2 + 1] = l[g];
+                }
+            }
+        }
+        __threadfence();
+        __syncwarp();
+        int ticket = 0;
+        if (lane == 0) ticket = atomicAdd(&p.tickets[s * Hg + hg], 1);
+        ticket = __shfl_sync(kFull, ticket, 0);
+        if (ticket == nu - 1) {
+            if (lane == 0) p.tickets[s * Hg + hg] = 0;   // ready for the next launch
+            __threadfence();
+            const int u0 = unit - c;
+            for (int g = 0; g < GT; ++g)
+                merge_partials_row<D, BF16>(p, u0, nu, g, GT, (size_t)s * p.Hq + (size_t)hg * GT + g, lane);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- merge kernel (resident + offloaded)
+
+__global__ void merge_kernel(const MergeParams p) {
+    const int warps_per_block = blockDim.x >> 5;
+    const int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= p.rows) return;
+    const float m1 = p.res_ml[row * 2], l1 = p.res_ml[row * 2 + 1];
+    float m2 = p.run_ml[row * 2];
+    const float l2 = p.run_ml[row * 2 + 1];
+    if (!(l2 > 0.f)) m2 = kNegBig;
+    const float mm = fmaxf(l1 > 0.f ? m1 : kNegBig, m2);
+    const float a1 = l1 > 0.f ? exp2f(m1 - mm) : 0.f;
+    const float a2 = l2 > 0.f ? exp2f(m2 - mm) : 0.f;
+    const float ll = l1 * a1 + l2 * a2;
+    const float inv = ll > 0.f ? 1.f / ll : 0.f;
+    for (int e = lane; e < p.D; e += 32) {
+        const size_t idx = (size_t)row * p.D + e;
+        float x = 0.f;
+        if (l1 > 0.f) x += p.res_o[idx] * a1;
+        if (l2 > 0.f) x += p.run_o[idx] * a2;
+        x *= inv;
+        if (p.out_f32) p.out_f32[idx] = x;
+        if (p.out) {
+            uint16_t *o16 = reinterpret_cast<uint16_t *>(p.out) + idx;
+            if (p.bf16) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(x);
+                *o16 = *reinterpret_cast<const uint16_t *>(&h);
+            } else {
+                const __half h = __float2half_rn(x);
+                *o16 = *reinterpret_cast<const uint16_t *>(&h);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- table update, append, fill, gather
+
+__global__ void table_update_kernel(int32_t *table, const TableUpdateBatch b) {
+    for (int i = threadIdx.x; i < b.n; i += blockDim.x) table[b.index[i]] = b.value[i];
+}
+
+// One CTA per sequence: K and V rows of the new token go to slot len % BT of
+// block len / BT (HBM pool, or the sequence's tail slot when the block is
+// host-flagged); then the length is incremented.
+__global__ void append_kernel(const AppendParams p) {
+    const int s = blockIdx.x;
+    const int len = p.lens[s];
+    const int j = len / p.BT, slot = len % p.BT;
+    const int32_t e = p.table[(size_t)s * p.table_stride + j];
+    uint8_t *base = nullptr;
+    if (e != ISV_BLOCK_NONE) {
+        if (e & ISV_BLOCK_HOST_BIT) {
+            if (p.tail) base = p.tail + (uint64_t)s * p.block_bytes;
+        } else if (e >= 0 && e < p.n_pool_blocks) {
+            base = p.pool + (uint64_t)e * p.block_bytes;
+        }
+    }
+    const int row_bytes = p.D * 2;
+    const int row_vecs = row_bytes / 16;
+    const uint32_t tile_bytes = (uint32_t)p.BT * row_bytes;
+    const int n = 2 * p.Hkv * row_vecs;
+    if (base) {
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const int kv = i / (p.Hkv * row_vecs);
+            const int r = i - kv * (p.Hkv * row_vecs);
+            const int h = r / row_vecs, vec = r - h * row_vecs;
+            const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
+                                 ((size_t)s * p.Hkv + h) * row_bytes + vec * 16;
+            uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)slot * row_bytes + vec * 16;
+            *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+        }
+    } else if (threadIdx.x == 0) {
+        atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+    }
+    __syncthreads();   // every thread has read the old length
+    if (threadIdx.x == 0) p.lens[s] = len + 1;
+}
+
+// Where block j of sequence s lives for a reader/writer that sees `len`
+// tokens: HBM pool, tail slot (host-flagged newest block) or host pool.
+__device__ __forceinline__ uint8_t *block_base(int32_t e, int s, int j, int len, int BT, uint8_t *pool, uint8_t *tail,
+                                               uint8_t *host, int n_pool, int n_host, uint64_t bb) {
+    if (e == ISV_BLOCK_NONE) return nullptr;
+    if (e & ISV_BLOCK_HOST_BIT) {
+        const int id = e & (ISV_BLOCK_HOST_BIT - 1);
+        if (j == (len - 1) / BT) return tail ? tail + (uint64_t)s * bb : nullptr;
+        return (host && id < n_host) ? host + (uint64_t)id * bb : nullptr;
+    }
+    return (e >= 0 && e < n_pool) ? pool + (uint64_t)e * bb : nullptr;
+}
+
+__global__ void fill_kernel(const FillParams p) {
+    const int j = blockIdx.x, s = blockIdx.y;
+    const int len = p.lens[s];
+    if (j * p.BT >= len) return;
+    const int ntok = min(p.BT, len - j * p.BT);
+    const int32_t e = p.table[(size_t)s * p.table_stride + j];
+    uint8_t *base = block_base(e, s, j, len, p.BT, p.pool, p.tail, p.host, p.n_pool_blocks, p.n_host_blocks,
+                               p.block_bytes);
+    if (!base) {
+        if (threadIdx.x == 0) atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+        return;
+    }
+    const int row_bytes = p.D * 2, row_vecs = row_bytes / 16;
+    const uint32_t tile_bytes = (uint32_t)p.BT * row_bytes;
+    const int per_kv = p.Hkv * ntok * row_vecs;
+    for (int i = threadIdx.x; i < 2 * per_kv; i += blockDim.x) {
+        const int kv = i / per_kv;
+        int r = i - kv * per_kv;
+        const int h = r / (ntok * row_vecs);
+        r -= h * ntok * row_vecs;
+        const int t = r / row_vecs, vec = r - t * row_vecs;
+        const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
+                             (((size_t)s * p.T + (size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
+        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + vec * 16;
+        *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+    }
+}
+
+__global__ void gather_kernel(const GatherParams p) {
+    const int j = blockIdx.x;
+    if (j * p.BT >= p.len) return;
+    const int ntok = min(p.BT, p.len - j * p.BT);
+    const int32_t e = p.table[j];
+    const uint8_t *base =
+        block_base(e, p.seq, j, p.len, p.BT, const_cast<uint8_t *>(p.pool), const_cast<uint8_t *>(p.tail),
+                   const_cast<uint8_t *>(p.host), p.n_pool_blocks, p.n_host_blocks, p.block_bytes);
+    if (!base) {
+        if (threadIdx.x == 0) atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+        return;
+    }
+    const int row_bytes = p.D * 2, row_vecs = row_bytes / 16;
+    const uint32_t tile_bytes = (uint32_t)p.BT * row_bytes;
+    const int per_kv = p.Hkv * ntok * row_vecs;
+    for (int i = threadIdx.x; i < 2 * per_kv; i += blockDim.x) {
+        const int kv = i / per_kv;
+        int r = i - kv * per_kv;
+        const int h = r / (ntok * row_vecs);
+        r -= h * ntok * row_vecs;
+        const int t = r / row_vecs, vec = r - t * row_vecs;
+        const uint8_t *src = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + vec * 16;
+        uint8_t *dst = reinterpret_cast<uint8_t *>(kv ? p.v_out : p.k_out) +
+                       (((size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
+        *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+    }
+}
+
+// ---------------------------------------------------------------- dispatch
+
+typedef void (*DecodeFn)(const DecodeParams, const int);
+
+template <int D, int GT, bool BF16>
+DecodeFn pick_mode(int mode) {
+    return mode == MODE_RESIDENT ? decode_kernel<D, GT, 16, BF16, MODE_RESIDENT>
+                                 : decode_kernel<D, GT, 16, BF16, MODE_STAGED>;
+}
+template <int D, int GT>
+DecodeFn pick_dtype(bool bf16, int mode) {
+    return bf16 ? pick_mode<D, GT, true>(mode) : pick_mode<D, GT, false>(mode);
+}
+template <int D>
+DecodeFn pick_gt(int GT, bool bf16, int mode) {
+    switch (GT) {
+        case 1: return pick_dtype<D, 1>(bf16, mode);
+        case 2: return pick_dtype<D, 2>(bf16, mode);
+        case 4: return pick_dtype<D, 4>(bf16, mode);
+        default: return nullptr;
+    }
+}
+DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
+    if (BT != 16) return nullptr;
+    if (D == 64) return pick_gt<64>(GT, bf16, mode);
+    if (D == 128) return pick_gt<128>(GT, bf16, mode);
+    return nullptr;
+}
+
+}  // namespace
+
+size_t decode_smem_bytes(int D, int BT, int stages, int max_seqs, int mode) {
+    const size_t stage = 2ull * BT * D * 2;
+    size_t b = (size_t)kDecodeWarps * stages * (stage + 8 + 4 * M_WORDS);
+    if (mode == MODE_RESIDENT) b += (size_t)(max_seqs + 1) * 4;
+    return b;
+}
+
+cudaError_t decode_configure(int D, int GT, int BT, bool bf16, int mode, size_t smem) {
+    DecodeFn fn = pick(D, GT, BT, bf16, mode);
+    if (!fn) return cudaErrorInvalidValue;
+    return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+
+cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int BT, bool bf16, int mode, int grid,
+                          int stages, size_t smem, cudaStream_t st) {
+    DecodeFn fn = pick(D, GT, BT, bf16, mode);
+    if (!fn) return cudaErrorInvalidValue;
+    fn<<<grid, kDecodeWarps * 32, smem, st>>>(p, stages);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_table_update(int32_t *table, const TableUpdateBatch &b, cudaStream_t st) {
+    table_update_kernel<<<1, 256, 0, st>>>(table, b);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_append(const AppendParams &p, cudaStream_t st) {
+    append_kernel<<<p.n_seqs, 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fill(const FillParams &p, cudaStream_t st) {
+    dim3 grid(p.max_blocks, p.n_seqs);
+    fill_kernel<<<grid, 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather(const GatherParams &p, cudaStream_t st) {
+    const int nblk = (p.len + p.BT - 1) / p.BT;
+    if (nblk == 0) return cudaSuccess;
+    gather_kernel<<<nblk, 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_merge(const MergeParams &p, cudaStream_t st) {
+    const int wpb = 8;
+    merge_kernel<<<(p.rows + wpb - 1) / wpb, wpb * 32, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace isv

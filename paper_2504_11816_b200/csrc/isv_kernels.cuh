@@ -1,0 +1,116 @@
+// Kernel parameter blocks and launchers (sm_100a).  Host code fills the
+// structs with plain pointers and sizes; nothing here owns memory.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace isv {
+
+constexpr int kDecodeWarps = 8;          // consumer warps per CTA of the decode kernel
+constexpr int kMaxTableUpdates = 480;    // entries one update launch carries by value
+
+enum DecodeMode : int { MODE_RESIDENT = 0, MODE_STAGED = 1 };
+
+// One launch of the split decode kernel.
+//   MODE_RESIDENT: units are (sequence, kv head x pass, split of `U` logical
+//     blocks); the kernel walks the block table, reads HBM-pool blocks and a
+//     host-flagged newest block from its tail slot, skips other host blocks.
+//     Each (sequence, head group) is finished by whichever unit arrives last
+//     (ticket), which merges the splits' partials.
+//   MODE_STAGED: units are (chunk unit, kv head x pass) from the plan lists;
+//     blocks are read from the staging buffer; results are merged into the
+//     running state acc_o / acc_ml, which one unit per launch owns.
+struct DecodeParams {
+    const uint8_t *pool;        // resident: layer slab of the HBM pool; staged: staging buffer
+    const uint8_t *tail;        // resident: layer slab of tail slots (NULL when nothing is offloaded)
+    const int32_t *table;       // [n_seqs][table_stride]
+    const int32_t *lens;        // [n_seqs] tokens to attend
+    int32_t table_stride;
+    int32_t n_pool_blocks;      // bound for block ids (pool blocks, or slots in the staging buffer)
+    // staged mode lists
+    const int32_t *cu_seq;
+    const int32_t *cu_beg;
+    const int32_t *cu_end;
+    const int32_t *cblk;
+    int32_t cu_first;
+    int32_t cu_count;
+    // inputs / outputs
+    const void *q;              // [n_seqs][Hq][D] 16-bit
+    void *out;                  // [n_seqs][Hq][D] 16-bit or NULL
+    float *out_f32;             // [n_seqs][Hq][D] or NULL
+    // scratch
+    float *part_o;              // [units][GT][D]
+    float *part_ml;             // [units][GT][2]
+    int32_t *tickets;           // [n_seqs][Hkv*P], zero between launches
+    float *acc_o;               // [n_seqs][Hq][D]  unnormalised result (resident, !finalize) / running state (staged)
+    float *acc_ml;              // [n_seqs][Hq][2]
+    uint32_t *status;
+    int32_t n_seqs, Hq, Hkv, P, U;
+    int32_t finalize;           // resident: 1 = normalise and write out; 0 = leave (m, l, o) in acc_*
+    float scale_log2;           // log2(e) / sqrt(D)
+    uint64_t block_bytes;
+};
+
+struct TableUpdateBatch {
+    int32_t n;
+    int32_t index[kMaxTableUpdates];
+    int32_t value[kMaxTableUpdates];
+};
+
+struct AppendParams {
+    const void *k, *v;          // [n_seqs][Hkv][D]
+    uint8_t *pool;              // layer slab, HBM pool
+    uint8_t *tail;              // layer slab, tail slots (may be NULL)
+    const int32_t *table;
+    int32_t *lens;              // [n_seqs], incremented by the kernel
+    uint32_t *status;
+    int32_t table_stride, n_pool_blocks;
+    int32_t n_seqs, Hkv, D, BT;
+    uint64_t block_bytes;
+};
+
+struct FillParams {
+    const void *k, *v;          // [n_seqs][T][Hkv][D]
+    uint8_t *pool, *tail, *host; // layer slabs: HBM pool, tail slots, host pool (mapped)
+    const int32_t *table;
+    const int32_t *lens;        // [n_seqs] device
+    uint32_t *status;
+    int32_t table_stride, n_pool_blocks, n_host_blocks;
+    int32_t n_seqs, T, Hkv, D, BT, max_blocks;
+    uint64_t block_bytes;
+};
+
+struct GatherParams {
+    void *k_out, *v_out;        // [len][Hkv][D] device
+    const uint8_t *pool, *tail, *host;
+    const int32_t *table;       // row of the sequence
+    uint32_t *status;
+    int32_t seq, len, n_pool_blocks, n_host_blocks;
+    int32_t Hkv, D, BT;
+    uint64_t block_bytes;
+};
+
+struct MergeParams {
+    const float *res_o, *res_ml;    // resident result (m, l, o)
+    const float *run_o, *run_ml;    // offloaded running state; l == 0 means empty
+    void *out;
+    float *out_f32;
+    int32_t rows, D, bf16;
+};
+
+// Bytes of dynamic shared memory the decode kernel needs for `stages` ring
+// stages per warp.
+size_t decode_smem_bytes(int D, int BT, int stages, int max_seqs, int mode);
+
+// Launchers return the CUDA error of the launch.
+cudaError_t decode_configure(int D, int GT, int BT, bool bf16, int mode, size_t smem);
+cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int BT, bool bf16, int mode,
+                          int grid, int stages, size_t smem, cudaStream_t st);
+cudaError_t launch_table_update(int32_t *table, const TableUpdateBatch &b, cudaStream_t st);
+cudaError_t launch_append(const AppendParams &p, cudaStream_t st);
+cudaError_t launch_fill(const FillParams &p, cudaStream_t st);
+cudaError_t launch_gather(const GatherParams &p, cudaStream_t st);
+cudaError_t launch_merge(const MergeParams &p, cudaStream_t st);
+
+}  // namespace isv

@@ -1,0 +1,319 @@
+"""Parity of the CUDA path against the fp64 reference, through the C ABI.
+Needs a B200; every test here is marked gpu."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attn as oa
+from oracle import kv_model as km
+from paper_2504_11816_b200 import binding as B
+from paper_2504_11816_b200 import workloads as W
+
+from _harness import TOL, Harness, bits_to_dev, dev_to_bits, values
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name="s", layers=2, q_heads=4, kv_heads=4, head_dim=128, dtype="f16", batch=5, ctx=(1, 100), steps=3,
+          f=0.5, perm=0, seed=11):
+    return W.Workload(name, layers, q_heads, kv_heads, head_dim, dtype, batch, ctx[0], ctx[1], steps, 16, f, perm, seed)
+
+
+# ---------------------------------------------------------------- the Tiny configuration, every row
+
+def test_tiny_config_one_append_one_decode_all_rows():
+    w = W.CONFIGS["tiny"]
+    with Harness(w) as hz:
+        hz.fill()
+        table = B.isv_block_table_host(hz.h, w.batch)
+        # every other block of the 256-token prompt is host-resident
+        for s in range(w.batch):
+            assert [bool(e & B.ISV_BLOCK_HOST_BIT) for e in table[s, :16]] == [j % 2 == 1 for j in range(16)]
+        res = hz.step()
+        err = hz.check_step(res)
+        assert err <= TOL
+        hz.check_gather()
+        # 8 of the 17 blocks of each sequence crossed the host link
+        r, o, staged, n_chunks = B.isv_plan_bytes(hz.h, 0, w.batch)
+        assert o == 4 * 8 * 16 * w.kv_bytes_per_token and r == 4 * (257 - 128) * w.kv_bytes_per_token
+
+
+# ---------------------------------------------------------------- offload fraction, permutation, splits, chunks
+
+@pytest.mark.parametrize("f", [0.0, 0.25, 0.5, 0.75, 1.0])
+@pytest.mark.parametrize("perm", [0, 5])
+def test_parity_over_offload_fractions_with_ragged_lengths(f, perm):
+    lens = [1, 15, 16, 17, 31, 32, 33, 100, 257, 640]
+    w = small(batch=len(lens), steps=20, f=f, perm=perm, ctx=(1, 640), q_heads=4, kv_heads=4, head_dim=128)
+    with Harness(w, lens=lens) as hz:
+        hz.fill()
+        hz.check_gather()
+        for t in range(w.steps):
+            res = hz.step()
+            hz.check_step(res)
+            r, o, _, _ = B.isv_plan_bytes(hz.h, 0, w.batch)
+            assert (r, o) == km.layer_step_bytes(hz.cur.tolist(), f, 16, w.kv_bytes_per_token)
+        hz.check_gather()
+
+
+@pytest.mark.parametrize("split", [1, 2, 7, 64])
+@pytest.mark.parametrize("chunk_blocks", [1, 0])
+def test_result_does_not_depend_on_split_or_chunk_size(split, chunk_blocks):
+    lens = [700, 33, 512, 129]
+    outs = []
+    w = small(batch=4, steps=2, f=0.5, perm=3, ctx=(1, 700), layers=1, q_heads=8, kv_heads=8, head_dim=64)
+    block_bytes = 2 * w.kv_heads * 16 * w.head_dim * 2
+    with Harness(w, lens=lens, split_blocks=split, chunk_bytes=chunk_blocks * block_bytes) as hz:
+        hz.fill()
+        for t in range(w.steps):
+            res = hz.step()
+            hz.check_step(res)
+            outs.append(res[0][1])
+    # same inputs with the default configuration: results agree within the bound
+    with Harness(w, lens=lens) as hz:
+        hz.fill()
+        for t in range(w.steps):
+            res = hz.step()
+            assert np.max(np.abs(res[0][1] - outs[t])) <= TOL
+
+
+# ---------------------------------------------------------------- head grouping, head dim, dtype
+
+@pytest.mark.parametrize("q_heads,kv_heads", [(8, 8), (8, 4), (8, 2), (16, 2), (6, 2)])
+@pytest.mark.parametrize("head_dim", [64, 128])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_parity_over_head_grouping_head_dim_and_dtype(q_heads, kv_heads, head_dim, dtype):
+    lens = [300, 17, 64, 1]
+    w = small(batch=4, steps=2, f=0.5, perm=9, ctx=(1, 300), layers=1, q_heads=q_heads, kv_heads=kv_heads,
+              head_dim=head_dim, dtype=dtype, seed=21)
+    with Harness(w, lens=lens) as hz:
+        hz.fill()
+        for t in range(w.steps):
+            hz.check_step(hz.step())
+        hz.check_gather()
+
+
+def test_identical_query_heads_of_a_group_give_identical_outputs():
+    w = small(batch=2, steps=1, f=0.5, layers=1, q_heads=8, kv_heads=2, head_dim=128, ctx=(90, 90))
+    with Harness(w) as hz:
+        hz.fill()
+        k, v, q = W.host_step(w, hz.rng)
+        q[:] = np.repeat(q[:, ::4], 4, axis=1)           # heads 4g..4g+3 are copies
+        kd, vd, qd = (bits_to_dev(x, w.dtype) for x in (k, v, q))
+        of = torch.zeros((w.batch, w.q_heads, w.head_dim), device="cuda")
+        torch.cuda.synchronize()
+        B.isv_kv_append(hz.h, 0, kd, vd, w.batch)
+        B.isv_attn_decode(hz.h, 0, qd, None, of, None, None, w.batch)
+        B.isv_sync(hz.h)
+        o = of.cpu().numpy()
+        for g in range(2):
+            for i in range(1, 4):
+                assert np.array_equal(o[:, 4 * g], o[:, 4 * g + i])
+
+
+# ---------------------------------------------------------------- special cases of the method
+
+@pytest.mark.parametrize("f", [0.0, 1.0])
+def test_context_of_one_token_returns_v_exactly(f):
+    w = small(batch=3, steps=1, f=f, layers=1, q_heads=4, kv_heads=2, head_dim=64, ctx=(0, 0))
+    with Harness(w, lens=[0, 0, 0]) as hz:
+        hz.fill()
+        res = hz.step()                                   # the appended token is the whole context
+        q, of, o16 = res[0]
+        kb, vb = zip(*[hz.shadow.gathered(0, s) for s in range(w.batch)])
+        for s in range(w.batch):
+            for h in range(w.q_heads):
+                assert np.array_equal(o16[s, h], vb[s][0, h // 2])
+                assert np.array_equal(of[s, h].astype(np.float64), oa.to_f64(values(vb[s][0, h // 2], w.dtype)))
+
+
+def test_zero_query_gives_the_mean_of_v():
+    w = small(batch=2, steps=1, f=0.5, layers=1, q_heads=4, kv_heads=4, head_dim=128, ctx=(333, 333))
+    with Harness(w) as hz:
+        hz.fill()
+        k, v, q = W.host_step(w, hz.rng)
+        q[:] = 0
+        kd, vd, qd = (bits_to_dev(x, w.dtype) for x in (k, v, q))
+        of = torch.zeros((w.batch, w.q_heads, w.head_dim), device="cuda")
+        torch.cuda.synchronize()
+        B.isv_kv_append(hz.h, 0, kd, vd, w.batch)
+        B.isv_attn_decode(hz.h, 0, qd, None, of, None, None, w.batch)
+        B.isv_sync(hz.h)
+        hz.shadow.append(0, k, v)
+        for s in range(w.batch):
+            vb = oa.to_f64(values(hz.shadow.gathered(0, s)[1], w.dtype))
+            assert np.max(np.abs(of[s].cpu().numpy() - vb.mean(axis=0))) <= 1e-5
+
+
+def test_empty_sequences_yield_zeros_and_fewer_sequences_can_be_decoded():
+    w = small(batch=4, steps=1, f=0.5, layers=1, q_heads=4, kv_heads=4, head_dim=64, ctx=(0, 50))
+    with Harness(w, lens=[50, 0, 20, 0]) as hz:
+        hz.fill()
+        _, _, q = W.host_step(w, hz.rng)
+        qd = bits_to_dev(q, w.dtype)
+        of = torch.full((w.batch, w.q_heads, w.head_dim), 7.0, device="cuda")
+        torch.cuda.synchronize()
+        B.isv_attn_decode(hz.h, 0, qd, None, of, None, None, w.batch)
+        B.isv_sync(hz.h)
+        o = of.cpu().numpy()
+        assert np.all(o[1] == 0) and np.all(o[3] == 0)
+        ref = hz.reference(0, q, seqs=[0, 2])
+        assert np.max(np.abs(o[[0, 2]] - ref)) <= TOL
+        # only the first sequence
+        of2 = torch.full((w.batch, w.q_heads, w.head_dim), 7.0, device="cuda")
+        torch.cuda.synchronize()
+        B.isv_attn_decode(hz.h, 0, qd, None, of2, None, None, 1)
+        B.isv_sync(hz.h)
+        o2 = of2.cpu().numpy()
+        assert np.max(np.abs(o2[0] - ref[0])) <= TOL and np.all(o2[1:] == 7.0)
+
+
+def test_unused_slots_may_hold_nan_patterns():
+    # fill every block with NaN bit patterns first, then reset and load short real data into the same blocks
+    lens = [5, 21, 40]
+    w = small(batch=3, steps=4, f=0.5, layers=1, q_heads=4, kv_heads=4, head_dim=128, ctx=(1, 64))
+    with Harness(w, lens=lens) as hz:
+        T = 64
+        nan_bits = np.full((w.batch, T, w.kv_heads, w.head_dim), 0x7e00, np.uint16)
+        nd = bits_to_dev(nan_bits, w.dtype)
+        torch.cuda.synchronize()
+        B.isv_kv_fill(hz.h, 0, nd, nd, np.full(w.batch, T, np.int32), w.batch, T)
+        B.isv_kv_reset(hz.h)
+        hz.fill()
+        for t in range(w.steps):
+            hz.check_step(hz.step())
+        hz.check_gather()
+
+
+def test_explicit_table_and_lengths_pointers_are_honoured():
+    w = small(batch=3, steps=1, f=0.0, layers=1, q_heads=4, kv_heads=4, head_dim=64, ctx=(70, 70))
+    with Harness(w) as hz:
+        hz.fill()
+        _, _, q = W.host_step(w, hz.rng)
+        qd = bits_to_dev(q, w.dtype)
+        info = B.isv_kv_info(hz.h)
+        table = torch.from_numpy(B.isv_block_table_host(hz.h, w.batch)).cuda()
+        lens = torch.tensor([70, 33, 1], dtype=torch.int32, device="cuda")     # attend to prefixes
+        of = torch.zeros((w.batch, w.q_heads, w.head_dim), device="cuda")
+        torch.cuda.synchronize()
+        B.isv_attn_decode(hz.h, 0, qd, None, of, table, lens, w.batch)
+        B.isv_sync(hz.h)
+        K, V = [], []
+        for s, n in enumerate([70, 33, 1]):
+            kb, vb = hz.shadow.gathered(0, s)
+            K.append(values(kb[:n], w.dtype))
+            V.append(values(vb[:n], w.dtype))
+        ref = oa.attn_decode(values(q, w.dtype), K, V)
+        assert np.max(np.abs(of.cpu().numpy() - ref)) <= TOL
+        assert info.max_blocks_per_seq == table.shape[1]
+
+
+# ---------------------------------------------------------------- whole-step entry points and timing
+
+@pytest.mark.parametrize("f", [0.0, 0.5])
+def test_decode_step_entry_points_match_per_layer_calls(f):
+    w = small(batch=4, steps=3, f=f, perm=2, layers=3, q_heads=8, kv_heads=4, head_dim=128, ctx=(40, 200))
+    td = W.torch_dtype(w.dtype)
+    with Harness(w) as ha, Harness(w) as hb, Harness(w) as hc:
+        for hz in (ha, hb, hc):
+            hz.fill()
+        B.isv_set_timing(hb.h, True)
+        for t in range(w.steps):
+            res = ha.step()
+            ha.check_step(res)
+            # replay the same inputs through the whole-step calls
+            ks, vs, qs = [], [], []
+            for layer in range(w.layers):
+                k, v, q = W.host_step(w, hb.rng)
+                W.host_step(w, hc.rng)
+                ks.append(k); vs.append(v); qs.append(q)
+                assert np.array_equal(q, res[layer][0])
+            k_all, v_all, q_all = (np.stack(x) for x in (ks, vs, qs))
+            kd, vd, qd = (bits_to_dev(x, w.dtype) for x in (k_all, v_all, q_all))
+            od = torch.zeros((w.layers, w.batch, w.q_heads, w.head_dim), device="cuda", dtype=td)
+            torch.cuda.synchronize()
+            B.isv_decode_step(hb.h, qd, kd, vd, od, w.batch)
+            B.isv_sync(hb.h)
+            got = dev_to_bits(od)
+            for layer in range(w.layers):
+                assert np.array_equal(got[layer], res[layer][2])
+            # host-buffer variant
+            kp, vp, qp = (torch.from_numpy(x.view(np.int16)).pin_memory() for x in (k_all, v_all, q_all))
+            op = torch.zeros((w.layers, w.batch, w.q_heads, w.head_dim), dtype=torch.int16).pin_memory()
+            B.isv_decode_step_host(hc.h, qp, kp, vp, op, w.batch)
+            assert np.array_equal(op.numpy().view(np.uint16), got)
+            # timing query: byte counters follow the cache model, times are sane
+            st = B.isv_step_timing(hb.h, -1)
+            res_b, off_b = km.layer_step_bytes(ha.cur.tolist(), f, 16, w.kv_bytes_per_token)
+            assert st.bytes_resident == w.layers * res_b and st.bytes_offloaded == w.layers * off_b
+            assert st.bytes_appended == w.layers * w.batch * w.kv_bytes_per_token
+            assert st.status == 0 and st.total_ms > 0 and st.attn_resident_ms > 0 and st.append_ms > 0
+            assert (st.h2d_ms > 0) == (off_b > 0) and (st.n_chunks > 0) == (off_b > 0)
+            assert st.total_ms >= st.attn_resident_ms
+            one = B.isv_step_timing(hb.h, 1)
+            assert one.bytes_resident == res_b and one.total_ms <= st.total_ms + 1e-3
+
+
+def test_link_probe_reports_plausible_rates():
+    h2d, d2h = B.isv_link_probe(256 << 20, 3)
+    assert 1.0 < h2d < 500.0 and 1.0 < d2h < 500.0
+
+
+# ---------------------------------------------------------------- full-size launch configuration, sampled rows
+
+def test_full_size_c2_shape_sampled_rows():
+    """Llama-2-7B-shaped decode batch (32 sequences x 32 heads x 128, context 1024, everything
+    resident) in the launch configuration the benchmark times; two layers; sampled rows are
+    compared with the reference, which is computed from the generator's own tensors."""
+    w = W.CONFIGS["c2"].with_(layers=2, steps=17)
+    td = W.torch_dtype(w.dtype)
+    h = B.isv_kv_alloc(**B.desc_from_workload(w))
+    try:
+        gen = W.device_generator(w)
+        lens = W.prompt_lens(w)
+        T = int(lens.max())
+        sample = [(0, 0), (0, 31), (13, 7), (31, 0), (31, 31), (5, 16), (22, 9), (17, 30)]
+        seqs = sorted({s for s, _ in sample})
+        Kh = {}   # (layer, seq) -> list of [n, Hkv, d] bit arrays
+        Vh = {}
+        for layer in range(w.layers):
+            k = W.device_normal(gen, (w.batch, T, w.kv_heads, w.head_dim), w.dtype)
+            v = W.device_normal(gen, (w.batch, T, w.kv_heads, w.head_dim), w.dtype)
+            torch.cuda.synchronize()
+            B.isv_kv_fill(h, layer, k, v, lens, w.batch, T)
+            for s in seqs:
+                Kh[(layer, s)] = [dev_to_bits(k[s])]
+                Vh[(layer, s)] = [dev_to_bits(v[s])]
+            del k, v
+        worst = 0.0
+        for t in range(w.steps):
+            q = W.device_normal(gen, (w.layers, w.batch, w.q_heads, w.head_dim), w.dtype)
+            k = W.device_normal(gen, (w.layers, w.batch, w.kv_heads, w.head_dim), w.dtype)
+            v = W.device_normal(gen, (w.layers, w.batch, w.kv_heads, w.head_dim), w.dtype)
+            out = torch.zeros_like(q)
+            torch.cuda.synchronize()
+            B.isv_decode_step(h, q, k, v, out, w.batch)
+            B.isv_sync(h)
+            for layer in range(w.layers):
+                for s in seqs:
+                    Kh[(layer, s)].append(dev_to_bits(k[layer, s])[None])
+                    Vh[(layer, s)].append(dev_to_bits(v[layer, s])[None])
+            if t in (0, 15, 16):          # 1025, 1040 (block just filled) and 1041 tokens
+                ob = dev_to_bits(out)
+                qb = dev_to_bits(q)
+                for layer in range(w.layers):
+                    for s, hd in sample:
+                        Ks = values(np.concatenate(Kh[(layer, s)]), w.dtype)[:, hd:hd + 1]
+                        Vs = values(np.concatenate(Vh[(layer, s)]), w.dtype)[:, hd:hd + 1]
+                        ref = oa.attn_decode(values(qb[layer, s:s + 1, hd:hd + 1], w.dtype), [Ks], [Vs])[0, 0]
+                        got = oa.to_f64(values(ob[layer, s, hd], w.dtype))
+                        worst = max(worst, float(np.max(np.abs(got - ref))))
+        assert worst <= TOL, worst
+        # gathers of a sampled sequence are bit-exact
+        n = int(lens[13]) + w.steps
+        kh = np.zeros((n, w.kv_heads, w.head_dim), np.uint16)
+        vh = np.zeros_like(kh)
+        assert B.isv_kv_gather(h, 1, 13, kh, vh) == n
+        assert np.array_equal(kh, np.concatenate(Kh[(1, 13)])) and np.array_equal(vh, np.concatenate(Vh[(1, 13)]))
+    finally:
+        B.isv_kv_free(h)
