@@ -303,8 +303,9 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
     if (h->stages_res < 2 || h->stages_stg < 2)
         return bail(fail(ISV_EINVAL, "shared memory (%d bytes) too small for this shape", smem_limit));
     const bool bf16 = g.dtype == ISV_BF16;
-    CUB(decode_configure(g.D, g.GT, g.BT, bf16, MODE_RESIDENT, h->smem_res));
-    CUB(decode_configure(g.D, g.GT, g.BT, bf16, MODE_STAGED, h->smem_stg));
+    // the per-function limit is shared by all handles: always raise it to the device maximum
+    CUB(decode_configure(g.D, g.GT, g.BT, bf16, MODE_RESIDENT, (size_t)smem_limit));
+    CUB(decode_configure(g.D, g.GT, g.BT, bf16, MODE_STAGED, (size_t)smem_limit));
 
     if (desc->compute_stream) {
         h->s_compute = (cudaStream_t)desc->compute_stream;
