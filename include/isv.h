@@ -240,6 +240,54 @@ int isv_sync(isv_kv *h, uint32_t *status_out);
  * that T_trans^d's BW_cpu->gpu stands for.  Allocates and frees its buffers. */
 int isv_link_probe(uint64_t bytes, int32_t reps, double *h2d_gbs, double *d2h_gbs);
 
+/* ---- decode attention for callers that cannot allocate ------------------- */
+
+/* Size of the fixed device array that holds this entry point's scratch.  Every
+ * GPU on which the library is loaded keeps this much memory until the process
+ * exits, whether or not the entry point is ever called. */
+#define ISV_STATIC_SCRATCH_BYTES (8u << 20)
+
+/* (The paper has no counterpart for this call: it is a packaging variant of
+ * isv_attn_decode's resident kernel, added for deployment reasons.)
+ *
+ * Some callers may not call cudaMalloc: a serving process that has handed all
+ * of its GPU memory to a framework's caching allocator, a latency-critical
+ * loop in which an allocation would stall the device, a plugin that is given
+ * pointers and a stream and nothing else.  This call is for them.  It makes no
+ * cudaMalloc / cudaFree / cudaHostAlloc and uses no allocating library call;
+ * it needs no handle.  The caller owns and passes every buffer:
+ *   kv_pool_dev      KV pool in the library's layout,
+ *                    [n_pool_blocks][K|V][kv_heads][block_tokens][head_dim], 16-bit
+ *   block_table_dev  int32 [n_seqs][table_stride]: pool block ids in logical
+ *                    order (ISV_BLOCK_NONE or host-flagged entries are skipped;
+ *                    ids outside the pool are skipped and flagged)
+ *   seq_lens_dev     int32 [n_seqs]: tokens to attend; at most
+ *                    max_blocks_per_seq * block_tokens each (not checked on the
+ *                    device: a larger length overruns the scratch)
+ *   q_dev            [n_seqs][q_heads][head_dim] 16-bit
+ *   out_dev / out_f32_dev   same shape, 16-bit / fp32; either may be NULL, not both
+ *   status_dev       optional uint32 the kernel ORs ISV_STATUS_* bits into
+ *                    (the caller clears it); NULL = not reported
+ *   stream           cudaStream_t the work is enqueued on (asynchronous)
+ * split_blocks: KV blocks per split, 0 = 8.
+ * The split kernel's partial results and arrival counters live in one fixed
+ * device array of ISV_STATIC_SCRATCH_BYTES.  A shape whose scratch
+ *   n_seqs * q_heads * ceil(max_blocks_per_seq / split_blocks) * (head_dim + 2) * 4 B (+ counters)
+ * does not fit is refused with ISV_ECAPACITY and a message; nothing runs then.
+ * All calls on a GPU share that array and it keeps the previous call's
+ * contents; each call zeroes the counters it needs on `stream` first.  Two
+ * calls whose GPU work overlaps (different streams, or different threads
+ * without ordering) race on it: order them on one stream or with events.
+ * The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress) and the device limits; make that first call with the
+ * device current and before starting any stream capture. */
+int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_blocks,
+                           const int32_t *block_table_dev, int32_t table_stride,
+                           const int32_t *seq_lens_dev, int32_t n_seqs, int32_t max_blocks_per_seq,
+                           int32_t q_heads, int32_t kv_heads, int32_t head_dim, int32_t block_tokens,
+                           int32_t dtype, int32_t split_blocks, const void *q_dev, void *out_dev,
+                           float *out_f32_dev, uint32_t *status_dev, void *stream);
+
 /* Text of the calling thread's last error; valid until its next call. */
 const char *isv_last_error(void);
 

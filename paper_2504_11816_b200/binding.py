@@ -36,7 +36,7 @@ EXPORTS = [
     "isv_attn_decode", "isv_decode_step", "isv_decode_step_host", "isv_kv_gather",
     "isv_block_table_dev", "isv_seq_lens_dev", "isv_block_table_host", "isv_seq_lens_host",
     "isv_plan_bytes", "isv_set_timing", "isv_step_timing", "isv_sync", "isv_link_probe",
-    "isv_last_error",
+    "isv_attn_decode_static", "isv_last_error",
 ]
 
 
@@ -123,6 +123,8 @@ def lib():
     L.isv_step_timing.argtypes = [vp, i32, P(StepTimes)]
     L.isv_sync.argtypes = [vp, P(ctypes.c_uint32)]
     L.isv_link_probe.argtypes = [u64, i32, P(ctypes.c_double), P(ctypes.c_double)]
+    L.isv_attn_decode_static.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp, vp,
+                                         vp, vp]
     L.isv_last_error.argtypes = []
     L.isv_last_error.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -263,6 +265,22 @@ def isv_link_probe(nbytes: int = 1 << 30, reps: int = 10):
     a, b = ctypes.c_double(0), ctypes.c_double(0)
     _check(lib().isv_link_probe(nbytes, reps, ctypes.byref(a), ctypes.byref(b)))
     return a.value, b.value
+
+
+ISV_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def isv_attn_decode_static(kv_pool, n_pool_blocks: int, block_table, table_stride: int, seq_lens, n_seqs: int,
+                           max_blocks_per_seq: int, q_heads: int, kv_heads: int, head_dim: int, block_tokens: int,
+                           dtype: int, split_blocks: int, q, out, out_f32, status=None, stream: int = 0):
+    """Decode attention over a caller-owned, all-resident paged KV pool without any
+    allocation by the library (for callers that may not call cudaMalloc: see
+    ``include/isv.h``).  Scratch is a fixed 8 MiB device array shared by all calls;
+    shapes that need more raise ``IsvError`` with code ``ISV_ECAPACITY``."""
+    _check(lib().isv_attn_decode_static(_ptr(kv_pool), n_pool_blocks, _ptr(block_table), table_stride,
+                                        _ptr(seq_lens), n_seqs, max_blocks_per_seq, q_heads, kv_heads, head_dim,
+                                        block_tokens, dtype, split_blocks, _ptr(q), _ptr(out), _ptr(out_f32),
+                                        _ptr(status), stream or None))
 
 
 def desc_from_workload(w, **overrides) -> dict:

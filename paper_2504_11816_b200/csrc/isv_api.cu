@@ -264,6 +264,11 @@ int upload_plan(isv_kv *h, const OffPlan &pl, PlanSlot **out) {
 
 }  // namespace
 
+// Lets the library's other translation units record the calling thread's last error.
+namespace isv {
+int set_error(int code, const char *msg) { return fail(code, "%s", msg); }
+}  // namespace isv
+
 // =========================================================================== C ABI
 
 extern "C" {
