@@ -180,7 +180,7 @@ def workload_config(w, args, info):
          "offload_frac": w.offload_frac, "batch": w.batch, "layers": w.layers, "accumulate": "f32",
          "l2": "KV read per layer-step exceeds L2 (inputs larger than L2)", "parallelism": "replicas"}
     if info is not None:
-        c.update({"phys_layers": info.phys_layers, "split_blocks": info.split_blocks,
+        c.update({"phys_layers": info.phys_layers, "max_ctas": info.max_ctas,
                   "chunk_bytes": info.chunk_bytes, "ring_depth": info.ring_depth})
     return c
 
@@ -410,6 +410,7 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--offload", type=float, default=None)
     ap.add_argument("--phys-layers", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=None, help="override the layer count (small profiling cases)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -417,6 +418,8 @@ def main():
     w = W.CONFIGS[args.workload]
     if args.offload is not None:
         w = w.with_(offload_frac=args.offload)
+    if args.layers is not None:
+        w = w.with_(layers=args.layers)
     if args.steps is None:
         args.steps = 64 if args.impl == "ours" and w.offload_frac == 0 else (5 if args.impl == "reference" else 4)
     if args.warmup < 0 or args.steps < 1:

@@ -83,7 +83,9 @@ typedef struct {
                                  /* follow a seeded permutation (host pool ids stay compact)    */
     uint64_t chunk_bytes;        /* staging chunk size; 0 = 32 MiB                              */
     int32_t  ring_depth;         /* staging ring buffers; 0 = 3                                 */
-    int32_t  split_blocks;       /* KV blocks per split of the resident kernel; 0 = 8           */
+    int32_t  max_ctas;           /* cap on the resident kernel's grid; 0 = one CTA per SM.      */
+                                 /* The KV blocks are cut evenly over the grid's warps, so this */
+                                 /* also sets into how many splits a sequence falls             */
     int32_t  plan_only;          /* 1 = host bookkeeping only: no CUDA call is made, no memory  */
                                  /* is allocated, compute entry points return ISV_ENODEVICE     */
     void    *compute_stream;     /* cudaStream_t to enqueue on, or NULL = library creates one   */
@@ -101,9 +103,9 @@ typedef struct {
     int32_t  host_blocks_used;
     uint64_t hbm_pool_bytes;     /* all physical layers, tail slots included                    */
     uint64_t host_pool_bytes;    /* all physical layers                                         */
-    uint64_t scratch_bytes;      /* partials, running state, staging ring                       */
+    uint64_t scratch_bytes;      /* split partials, running state, staging ring                 */
     int32_t  phys_layers;
-    int32_t  split_blocks;
+    int32_t  max_ctas;
     int32_t  ring_depth;
     int32_t  sm_count;
     uint64_t chunk_bytes;
@@ -262,17 +264,18 @@ int isv_link_probe(uint64_t bytes, int32_t reps, double *h2d_gbs, double *d2h_gb
  *                    order (ISV_BLOCK_NONE or host-flagged entries are skipped;
  *                    ids outside the pool are skipped and flagged)
  *   seq_lens_dev     int32 [n_seqs]: tokens to attend; at most
- *                    max_blocks_per_seq * block_tokens each (not checked on the
- *                    device: a larger length overruns the scratch)
+ *                    max_blocks_per_seq * block_tokens each (the table rows must
+ *                    cover them)
  *   q_dev            [n_seqs][q_heads][head_dim] 16-bit
  *   out_dev / out_f32_dev   same shape, 16-bit / fp32; either may be NULL, not both
  *   status_dev       optional uint32 the kernel ORs ISV_STATUS_* bits into
  *                    (the caller clears it); NULL = not reported
  *   stream           cudaStream_t the work is enqueued on (asynchronous)
- * split_blocks: KV blocks per split, 0 = 8.
+ * max_ctas: cap on the kernel's grid, 0 = one CTA per SM.
  * The split kernel's partial results and arrival counters live in one fixed
  * device array of ISV_STATIC_SCRATCH_BYTES.  A shape whose scratch
- *   n_seqs * q_heads * ceil(max_blocks_per_seq / split_blocks) * (head_dim + 2) * 4 B (+ counters)
+ *   n_seqs * (q_heads / heads per warp) * 4 B of counters
+ *   + 2 * warps in the grid * heads per warp * (head_dim + 2) * 4 B of partials
  * does not fit is refused with ISV_ECAPACITY and a message; nothing runs then.
  * All calls on a GPU share that array and it keeps the previous call's
  * contents; each call zeroes the counters it needs on `stream` first.  Two
@@ -285,7 +288,7 @@ int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_blocks,
                            const int32_t *block_table_dev, int32_t table_stride,
                            const int32_t *seq_lens_dev, int32_t n_seqs, int32_t max_blocks_per_seq,
                            int32_t q_heads, int32_t kv_heads, int32_t head_dim, int32_t block_tokens,
-                           int32_t dtype, int32_t split_blocks, const void *q_dev, void *out_dev,
+                           int32_t dtype, int32_t max_ctas, const void *q_dev, void *out_dev,
                            float *out_f32_dev, uint32_t *status_dev, void *stream);
 
 /* Text of the calling thread's last error; valid until its next call. */

@@ -54,7 +54,7 @@ class KvDesc(ctypes.Structure):
         ("block_tokens", ctypes.c_int32), ("dtype", ctypes.c_int32), ("offload_frac", ctypes.c_float),
         ("max_seqs", ctypes.c_int32), ("max_tokens_per_seq", ctypes.c_int32),
         ("perm_seed", ctypes.c_uint64), ("chunk_bytes", ctypes.c_uint64),
-        ("ring_depth", ctypes.c_int32), ("split_blocks", ctypes.c_int32), ("plan_only", ctypes.c_int32),
+        ("ring_depth", ctypes.c_int32), ("max_ctas", ctypes.c_int32), ("plan_only", ctypes.c_int32),
         ("compute_stream", ctypes.c_void_p),
     ]
 
@@ -67,7 +67,7 @@ class KvInfo(ctypes.Structure):
         ("host_blocks_used", ctypes.c_int32),
         ("hbm_pool_bytes", ctypes.c_uint64), ("host_pool_bytes", ctypes.c_uint64),
         ("scratch_bytes", ctypes.c_uint64),
-        ("phys_layers", ctypes.c_int32), ("split_blocks", ctypes.c_int32),
+        ("phys_layers", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
         ("ring_depth", ctypes.c_int32), ("sm_count", ctypes.c_int32),
         ("chunk_bytes", ctypes.c_uint64), ("kernel_launches", ctypes.c_uint64),
     ]
@@ -272,14 +272,14 @@ ISV_STATIC_SCRATCH_BYTES = 8 << 20
 
 def isv_attn_decode_static(kv_pool, n_pool_blocks: int, block_table, table_stride: int, seq_lens, n_seqs: int,
                            max_blocks_per_seq: int, q_heads: int, kv_heads: int, head_dim: int, block_tokens: int,
-                           dtype: int, split_blocks: int, q, out, out_f32, status=None, stream: int = 0):
+                           dtype: int, max_ctas: int, q, out, out_f32, status=None, stream: int = 0):
     """Decode attention over a caller-owned, all-resident paged KV pool without any
     allocation by the library (for callers that may not call cudaMalloc: see
     ``include/isv.h``).  Scratch is a fixed 8 MiB device array shared by all calls;
     shapes that need more raise ``IsvError`` with code ``ISV_ECAPACITY``."""
     _check(lib().isv_attn_decode_static(_ptr(kv_pool), n_pool_blocks, _ptr(block_table), table_stride,
                                         _ptr(seq_lens), n_seqs, max_blocks_per_seq, q_heads, kv_heads, head_dim,
-                                        block_tokens, dtype, split_blocks, _ptr(q), _ptr(out), _ptr(out_f32),
+                                        block_tokens, dtype, max_ctas, _ptr(q), _ptr(out), _ptr(out_f32),
                                         _ptr(status), stream or None))
 
 

@@ -157,8 +157,8 @@ int dev_alloc(void **p, size_t bytes, uint64_t *tally, const char *what) {
 
 int pick_stages(const Geometry &g, int mode, int smem_limit, size_t *smem_out) {
     int best = 0;
-    for (int st = 2; st <= 8; ++st) {
-        const size_t b = decode_smem_bytes(g.D, g.BT, st, g.max_seqs, mode);
+    for (int st = 2; st <= 12; ++st) {
+        const size_t b = decode_smem_bytes(g.D, g.BT, g.GT, st, g.max_seqs, mode);
         if (b <= (size_t)smem_limit) { best = st; *smem_out = b; }
     }
     return best;
@@ -350,9 +350,10 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
     CUB(cudaMemset(h->status_dev, 0, 4));
     // scratch
     const size_t rows = (size_t)g.max_seqs * g.Hq;
-    const size_t splits = (size_t)(g.NB + g.U - 1) / g.U;
-    if ((rc = dev_alloc((void **)&h->part_o, rows * splits * g.D * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
-    if ((rc = dev_alloc((void **)&h->part_ml, rows * splits * 2 * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
+    const int max_grid = g.max_ctas > 0 ? std::min(g.max_ctas, h->sm_count) : h->sm_count;
+    const size_t slots = 2ull * max_grid * decode_warps(g.GT) * g.GT;   // two partials per warp and query head
+    if ((rc = dev_alloc((void **)&h->part_o, slots * g.D * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
+    if ((rc = dev_alloc((void **)&h->part_ml, slots * 2 * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
     if ((rc = dev_alloc((void **)&h->tickets, (size_t)g.max_seqs * g.Hkv * g.P * 4, &h->scratch_bytes, "tickets"))) return bail(rc);
     CUB(cudaMemset(h->tickets, 0, (size_t)g.max_seqs * g.Hkv * g.P * 4));
     if (g.host_cap > 0) {
@@ -437,7 +438,7 @@ int isv_kv_info(isv_kv *h, isv_kv_info_t *o) {
     o->host_pool_bytes = (uint64_t)h->g.phys_layers * h->g.host_cap * h->g.block_bytes;
     o->scratch_bytes = h->scratch_bytes;
     o->phys_layers = h->g.phys_layers;
-    o->split_blocks = h->g.U;
+    o->max_ctas = h->g.max_ctas;
     o->ring_depth = h->g.ring;
     o->sm_count = h->sm_count;
     o->chunk_bytes = h->g.chunk_bytes;
@@ -569,6 +570,7 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *o
     if (n_seqs == 0) return ISV_OK;
     const bool bf16 = g.dtype == ISV_BF16;
     const int Hg = g.Hkv * g.P;
+    const int nw = decode_warps(g.GT);
     const OffPlan &pl = h->bm.plan(layer, n_seqs);
     const bool offloaded = !pl.chunks.empty();
     const int phys = layer % g.phys_layers;
@@ -591,7 +593,7 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *o
     base.table_stride = g.NB;
     base.q = q;
     base.status = h->status_dev;
-    base.n_seqs = n_seqs; base.Hq = g.Hq; base.Hkv = g.Hkv; base.P = g.P; base.U = g.U;
+    base.n_seqs = n_seqs; base.Hq = g.Hq; base.Hkv = g.Hkv; base.P = g.P;
     base.block_bytes = g.block_bytes;
     base.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)g.D));
 
@@ -628,7 +630,7 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *o
             p.acc_o = h->run_o;
             p.acc_ml = h->run_ml;
             const long long nu2 = (long long)p.cu_count * Hg;
-            const int grid = (int)std::max<long long>(1, std::min<long long>(h->sm_count, (nu2 + kDecodeWarps - 1) / kDecodeWarps));
+            const int grid = (int)std::max<long long>(1, std::min<long long>(h->sm_count, (nu2 + nw - 1) / nw));
             CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_STAGED, grid, h->stages_stg, h->smem_stg, h->s_off));
             ++h->launches;
             CU(cudaEventRecord(h->ev_freed[r], h->s_off));
@@ -653,12 +655,11 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *o
         p.part_o = h->part_o; p.part_ml = h->part_ml; p.tickets = h->tickets;
         p.acc_o = h->res_o; p.acc_ml = h->res_ml;
         p.finalize = offloaded ? 0 : 1;
-        long long nu = 0;
-        for (int s = 0; s < n_seqs; ++s) {
-            const int nblk = (h->bm.length(layer, s) + g.BT - 1) / g.BT;
-            nu += (long long)std::max(1, (nblk + g.U - 1) / g.U) * Hg;
-        }
-        const int grid = (int)std::max<long long>(1, std::min<long long>(h->sm_count, (nu + kDecodeWarps - 1) / kDecodeWarps));
+        long long nu = 0;   // KV blocks in the flat work list
+        for (int s = 0; s < n_seqs; ++s)
+            nu += (long long)std::max(1, (h->bm.length(layer, s) + g.BT - 1) / g.BT) * Hg;
+        const int cap = g.max_ctas > 0 ? std::min(g.max_ctas, h->sm_count) : h->sm_count;
+        const int grid = (int)std::max<long long>(1, std::min<long long>(cap, (nu + nw - 1) / nw));
         if (le) CU(cudaEventRecord(le->r0, h->s_compute));
         CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_RESIDENT, grid, h->stages_res, h->smem_res, h->s_compute));
         ++h->launches;

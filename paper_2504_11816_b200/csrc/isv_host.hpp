@@ -23,7 +23,7 @@ struct Geometry {
     int G = 0;                     // query heads per KV head
     int GT = 0;                    // query heads handled together by one warp
     int P = 0;                     // passes over a KV head = G / GT
-    int U = 0;                     // KV blocks per split
+    int max_ctas = 0;              // cap on the decode kernel's grid (0 = one CTA per SM)
     uint32_t tile_bytes = 0;       // one (block, K|V, head) tile
     uint64_t block_bytes = 0;      // 2 * Hkv * tile_bytes
     uint64_t kappa = 0;            // KV bytes per token per layer
@@ -292,8 +292,9 @@ inline const char *make_geometry(const isv_kv_desc &d, Geometry *out) {
     if (hbm_cap >= ISV_BLOCK_HOST_BIT || host_cap >= ISV_BLOCK_HOST_BIT) return "too many blocks";
     g.hbm_cap = (int)hbm_cap;
     g.host_cap = (int)host_cap;
-    g.U = d.split_blocks == 0 ? 8 : d.split_blocks;
-    if (g.U < 1) return "split_blocks must be >= 1";
+    if (d.max_ctas < 0) return "max_ctas must be >= 0";
+    g.max_ctas = d.max_ctas;
+    if ((long long)g.max_seqs * g.NB * g.Hkv * g.P >= (1ll << 31)) return "max_seqs * blocks * heads too large";
     g.chunk_bytes = d.chunk_bytes == 0 ? (32ull << 20) : d.chunk_bytes;
     g.chunk_blocks = (int)std::max<uint64_t>(1, g.chunk_bytes / g.block_bytes);
     g.chunk_bytes = (uint64_t)g.chunk_blocks * g.block_bytes;

@@ -97,24 +97,26 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
     }
 }
 
-// ---------------------------------------------------------------- one K/V tile
+// ---------------------------------------------------------------- one K tile, one V tile
 
 // Lane layout inside a warp: grp = lane / 8 owns tokens grp, grp+4, ... of the
 // tile; sub = lane % 8 owns head-dim elements [v*64 + sub*8, +8) for v < D/64.
 // Each group keeps its own running (m, l, o); groups are merged at unit end.
+
+// Scores of the tile's tokens against the GT query heads (log2 domain, q is
+// pre-scaled), and the running maximum brought up to date (o and l rescaled).
 template <int D, int GT, int BT, bool BF16>
-__device__ __forceinline__ void tile_compute(const uint8_t *sK, const uint8_t *sV, int ntok, int grp, int sub,
-                                             const float (&q)[GT][D / 8], float (&o)[GT][D / 8], float (&m)[GT],
-                                             float (&l)[GT]) {
+__device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp, int sub,
+                                            const float (&q)[GT][D / 8], float (&sc)[BT / 4][GT],
+                                            float (&o)[GT][D / 8], float (&m)[GT], float (&l)[GT]) {
     constexpr int NV = D / 64, NQ = BT / 4, ROW = D * 2;
-    float sc[NQ][GT];
 #pragma unroll
     for (int i = 0; i < NQ; ++i) {
         const int t = 4 * i + grp;
         const uint4 *kp = reinterpret_cast<const uint4 *>(sK + t * ROW) + sub;
-        float acc[GT];
+        float a0[GT], a1[GT];   // two chains per dot product
 #pragma unroll
-        for (int g = 0; g < GT; ++g) acc[g] = 0.f;
+        for (int g = 0; g < GT; ++g) a0[g] = a1[g] = 0.f;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             float kf[8];
@@ -122,11 +124,14 @@ __device__ __forceinline__ void tile_compute(const uint8_t *sK, const uint8_t *s
 #pragma unroll
             for (int g = 0; g < GT; ++g)
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[g] = fmaf(q[g][v * 8 + e], kf[e], acc[g]);
+                for (int e = 0; e < 8; e += 2) {
+                    a0[g] = fmaf(q[g][v * 8 + e], kf[e], a0[g]);
+                    a1[g] = fmaf(q[g][v * 8 + e + 1], kf[e + 1], a1[g]);
+                }
         }
 #pragma unroll
         for (int g = 0; g < GT; ++g) {
-            float a = acc[g];
+            float a = a0[g] + a1[g];
             a += __shfl_xor_sync(kFull, a, 4);
             a += __shfl_xor_sync(kFull, a, 2);
             a += __shfl_xor_sync(kFull, a, 1);
@@ -146,6 +151,14 @@ __device__ __forceinline__ void tile_compute(const uint8_t *sK, const uint8_t *s
             m[g] = mx;
         }
     }
+}
+
+// o += softmax weights x V for the tile whose scores are in sc.
+template <int D, int GT, int BT, bool BF16>
+__device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp, int sub,
+                                            const float (&sc)[BT / 4][GT], float (&o)[GT][D / 8],
+                                            const float (&m)[GT], float (&l)[GT]) {
+    constexpr int NV = D / 64, NQ = BT / 4, ROW = D * 2;
 #pragma unroll
     for (int i = 0; i < NQ; ++i) {
         const int t = 4 * i + grp;
@@ -195,22 +208,24 @@ __device__ __forceinline__ void store_row_grouped(void *out, float *out_f32, siz
     }
 }
 
-// Last-arriving unit of a (sequence, head group): combine the nu partials of
-// query head g.  Lane owns D/32 consecutive elements.
+// Last-arriving contributor of a (sequence, head group): combine the nc partials of
+// query head g in fixed order.  Lane owns D/32 consecutive elements.
 template <int D, bool BF16>
-__device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int u0, int nu, int g, int GT,
+__device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int wf, int wf_slot, int nc, int g, int GT,
                                                    size_t row, int lane) {
     constexpr int EPL = D / 32;
+    // contributor c is warp wf + c; the first one may have used its second slot, all others used their first
+    auto slot_of = [&](int c) { return c == 0 ? 2 * wf + wf_slot : 2 * (wf + c); };
     float mm = kNegBig;
-    for (int c = lane; c < nu; c += 32) mm = fmaxf(mm, __ldcg(&p.part_ml[((size_t)(u0 + c) * GT + g) * 2]));
+    for (int c = lane; c < nc; c += 32) mm = fmaxf(mm, __ldcg(&p.part_ml[((size_t)slot_of(c) * GT + g) * 2]));
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) mm = fmaxf(mm, __shfl_xor_sync(kFull, mm, d));
     float ll = 0.f;
     float acc[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-    for (int c = 0; c < nu; ++c) {
-        const size_t pr = (size_t)(u0 + c) * GT + g;
+    for (int c = 0; c < nc; ++c) {
+        const size_t pr = (size_t)slot_of(c) * GT + g;
         const float2 ml = __ldcg(reinterpret_cast<const float2 *>(&p.part_ml[pr * 2]));
         const float a = exp2f(ml.x - mm);
         ll += ml.y * a;
@@ -258,35 +273,43 @@ __device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int u0
 // ---------------------------------------------------------------- decode kernel
 
 // Stage metadata words written by the producing lane before it arms the stage.
-enum { M_UNIT = 0, M_SEQ, M_HG, M_C, M_NU, M_NTOK, M_LAST, M_WORDS = 8 };
+enum { M_SEG = 0, M_SEQ, M_HG, M_NTOK, M_FLAGS, M_NC, M_WF, M_WFSLOT, M_WORDS = 8 };
+enum { F_KIND_K = 0, F_KIND_V = 1, F_KIND_END = 2, F_KIND_MASK = 3, F_LAST = 4 };
 
-template <int D, int GT, int BT, bool BF16, int MODE>
-__global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const DecodeParams p, const int stages) {
+// A split whose partial has been stored but whose arrival has not been
+// published yet (publishing needs a fence; it is cheap once the stores have
+// landed, so it is done one unit later).
+struct PendingArrival {
+    int valid, ticket_idx, nc, wf, wf_slot;
+    size_t row0;
+};
+
+template <int D, int GT, int BT, bool BF16, int MODE, int NW>
+__global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p, const int stages) {
     constexpr uint32_t TILE = BT * D * 2;
-    constexpr uint32_t STAGE = 2 * TILE;
     constexpr int E = D / 8;
     extern __shared__ __align__(128) uint8_t smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int grp = lane >> 3, sub = lane & 7;
 
-    uint8_t *data = smem + (size_t)warp * stages * STAGE;
-    uint8_t *after_data = smem + (size_t)kDecodeWarps * stages * STAGE;
+    uint8_t *data = smem + (size_t)warp * stages * TILE;
+    uint8_t *after_data = smem + (size_t)NW * stages * TILE;
     uint64_t *bars = reinterpret_cast<uint64_t *>(after_data) + warp * stages;
-    int32_t *meta = reinterpret_cast<int32_t *>(after_data + (size_t)kDecodeWarps * stages * 8) +
-                    warp * stages * M_WORDS;
-    int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)kDecodeWarps * stages * (8 + 4 * M_WORDS));
+    int32_t *meta = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * 8) + warp * stages * M_WORDS;
+    int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * (8 + 4 * M_WORDS));
 
     const int Hg = p.Hkv * p.P;
     const uint64_t block_bytes = p.block_bytes;
 
-    // ---- unit count and this warp's contiguous range of units
-    int NU;
+    // ---- this warp's contiguous share of the work.  Resident mode: the flat space of KV blocks
+    // ordered by (sequence, head group, block), cut into equal ranges whatever the sequence lengths
+    // (an empty sequence counts as one block without tokens so that its zeros get written).
+    // Staged mode: whole (chunk unit, head group) items.
+    long long NU;
     if (MODE == MODE_RESIDENT) {
         for (int s = threadIdx.x; s < p.n_seqs; s += blockDim.x) {
             const int len = p.lens[s];
-            const int nblk = (len + BT - 1) / BT;
-            const int nu = max(1, (nblk + p.U - 1) / p.U);
-            ubase[s + 1] = nu * Hg;
+            ubase[s + 1] = max(1, (len + BT - 1) / BT) * Hg;
         }
         if (threadIdx.x == 0) ubase[0] = 0;
         __syncthreads();
@@ -307,13 +330,14 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
         __syncthreads();
         NU = ubase[p.n_seqs];
     } else {
-        NU = p.cu_count * Hg;
+        NU = (long long)p.cu_count * Hg;
     }
-    const long long nwt = (long long)gridDim.x * kDecodeWarps;
-    const long long gw = (long long)blockIdx.x * kDecodeWarps + warp;
-    int u_next = (int)((long long)NU * gw / nwt);
-    const int u_end = (int)((long long)NU * (gw + 1) / nwt);
-    if (u_next >= u_end) return;
+    // no more ranges than items, so that every participating warp owns at least one item
+    const long long nwt = min((long long)gridDim.x * NW, NU);
+    const int gw = blockIdx.x * NW + warp;
+    if (gw >= nwt) return;
+    int u_next = (int)(NU * gw / nwt);
+    const int u_end = (int)(NU * (gw + 1) / nwt);
 
     if (lane == 0) {
         for (int st = 0; st < stages; ++st) mbar_init(smem_u32(&bars[st]), 1);
@@ -322,12 +346,14 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
     __syncwarp();
 
     // ---- producer state (identical in all lanes except `ent`)
-    int pu_unit = -1, pu_s = 0, pu_hg = 0, pu_c = 0, pu_nu = 1;
+    int pu_seg = -1, pu_s = 0, pu_hg = 0, pu_nc = 1, pu_wf = 0, pu_wfslot = 0;
     int pu_len = 0, pu_jlast = -1, pu_j0 = 0, pu_n = 0;   // entries of the open unit: [pu_j0, pu_j0 + pu_n)
     int pu_batch = 0, pu_nbatch = 0, pu_base = 0;
     uint32_t pu_mask = 0;
     int32_t ent = ISV_BLOCK_NONE;
     bool pu_open = false, pu_done = false;
+    const uint8_t *pv_src = nullptr;    // V tile of the block whose K tile was just issued
+    int pv_ntok = 0, pv_flags = 0;
     int prod_stage = 0, inflight = 0;
     if (MODE == MODE_RESIDENT) {   // sequence of the first unit: largest s with ubase[s] <= u_next
         int lo = 0, hi = p.n_seqs - 1;
@@ -338,8 +364,30 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
         pu_s = lo;
     }
 
-    // Emits at most one stage (a tile, or an end-of-unit marker without data).
+    auto emit = [&](const uint8_t *src, int ntok, int flags) {   // one stage: a tile, or a marker without data
+        if (lane == 0) {
+            int32_t *mt = meta + prod_stage * M_WORDS;
+            mt[M_SEG] = pu_seg; mt[M_SEQ] = pu_s; mt[M_HG] = pu_hg; mt[M_NTOK] = ntok; mt[M_FLAGS] = flags;
+            mt[M_NC] = pu_nc; mt[M_WF] = pu_wf; mt[M_WFSLOT] = pu_wfslot;
+            const uint32_t bar = smem_u32(&bars[prod_stage]);
+            if (src) {
+                mbar_arrive_expect_tx(bar, TILE);
+                bulk_g2s(smem_u32(data + (size_t)prod_stage * TILE), src, TILE, bar);
+            } else {
+                mbar_arrive(bar);
+            }
+        }
+        prod_stage = (prod_stage + 1 == stages) ? 0 : prod_stage + 1;
+        ++inflight;
+    };
+
+    // Emits at most one stage.
     auto produce = [&]() {
+        if (pv_src) {   // second half of the current block
+            emit(pv_src, pv_ntok, pv_flags);
+            pv_src = nullptr;
+            return;
+        }
         while (true) {
             if (pu_mask != 0) {
                 const int i = __ffs(pu_mask) - 1;
@@ -357,19 +405,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
                     src = p.pool + (uint64_t)e * block_bytes;
                 }
                 const int kvh = pu_hg / p.P;
-                if (lane == 0) {
-                    int32_t *mt = meta + prod_stage * M_WORDS;
-                    mt[M_UNIT] = pu_unit; mt[M_SEQ] = pu_s; mt[M_HG] = pu_hg; mt[M_C] = pu_c;
-                    mt[M_NU] = pu_nu; mt[M_NTOK] = ntok; mt[M_LAST] = last ? 1 : 0;
-                    const uint32_t bar = smem_u32(&bars[prod_stage]);
-                    const uint32_t dst = smem_u32(data + (size_t)prod_stage * STAGE);
-                    mbar_arrive_expect_tx(bar, STAGE);
-                    bulk_g2s(dst, src + (uint64_t)kvh * TILE, TILE, bar);
-                    bulk_g2s(dst + TILE, src + (uint64_t)(p.Hkv + kvh) * TILE, TILE, bar);
-                }
+                pv_src = src + (uint64_t)(p.Hkv + kvh) * TILE;
+                pv_ntok = ntok;
+                pv_flags = F_KIND_V | (last ? F_LAST : 0);
+                emit(src + (uint64_t)kvh * TILE, ntok, F_KIND_K);
                 if (last) pu_open = false;
-                prod_stage = (prod_stage + 1 == stages) ? 0 : prod_stage + 1;
-                ++inflight;
                 return;
             }
             if (pu_open) {
@@ -401,39 +441,45 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
                     continue;
                 }
                 // no tile carried the end flag (or the unit is empty): explicit end marker
-                if (lane == 0) {
-                    int32_t *mt = meta + prod_stage * M_WORDS;
-                    mt[M_UNIT] = pu_unit; mt[M_SEQ] = pu_s; mt[M_HG] = pu_hg; mt[M_C] = pu_c;
-                    mt[M_NU] = pu_nu; mt[M_NTOK] = 0; mt[M_LAST] = 1;
-                    mbar_arrive(smem_u32(&bars[prod_stage]));
-                }
+                emit(nullptr, 0, F_KIND_END | F_LAST);
                 pu_open = false;
-                prod_stage = (prod_stage + 1 == stages) ? 0 : prod_stage + 1;
-                ++inflight;
                 return;
             }
             if (u_next >= u_end) { pu_done = true; return; }
-            // open the next unit
-            pu_unit = u_next++;
+            // open the next segment (resident) or unit (staged)
+            ++pu_seg;
             if (MODE == MODE_RESIDENT) {
-                while (pu_unit >= ubase[pu_s + 1]) ++pu_s;
+                const int x = u_next;
+                while (x >= ubase[pu_s + 1]) ++pu_s;
                 pu_len = p.lens[pu_s];
                 const int nblk = (pu_len + BT - 1) / BT;
-                pu_nu = max(1, (nblk + p.U - 1) / p.U);
-                const int r = pu_unit - ubase[pu_s];
-                pu_hg = r / pu_nu;
-                pu_c = r - pu_hg * pu_nu;
-                pu_j0 = pu_c * p.U;
-                pu_n = max(0, min(p.U, nblk - pu_j0));
+                const int nb = max(1, nblk);
+                const int r = x - ubase[pu_s];
+                pu_hg = r / nb;
+                pu_j0 = r - pu_hg * nb;
+                const int start = ubase[pu_s] + pu_hg * nb;           // flat range of this (sequence, head group)
+                const int seg_end = min(u_end, start + nb);
+                const int n = seg_end - x;
+                u_next = seg_end;
+                pu_n = nblk == 0 ? 0 : n;
                 pu_jlast = nblk - 1;
+                if (pu_j0 == 0 && n == nb) {
+                    pu_nc = 1;                                        // this warp holds all of it
+                } else {
+                    // warps whose ranges meet [start, start + nb): warp of index i is the largest w with NU*w/nwt <= i
+                    pu_wf = (int)((((long long)start + 1) * nwt - 1) / NU);
+                    const int wl = (int)((((long long)start + nb) * nwt - 1) / NU);
+                    pu_nc = wl - pu_wf + 1;
+                    pu_wfslot = (NU * pu_wf / nwt == start) ? 0 : 1;
+                }
             } else {
-                const int cu = p.cu_first + pu_unit / Hg;
-                pu_hg = pu_unit % Hg;
+                const int unit = u_next++;
+                const int cu = p.cu_first + unit / Hg;
+                pu_hg = unit % Hg;
                 pu_s = p.cu_seq[cu];
                 pu_j0 = p.cu_beg[cu];
                 pu_n = p.cu_end[cu] - pu_j0;
-                pu_c = 0;
-                pu_nu = 1;
+                pu_nc = 1;
             }
             pu_nbatch = (pu_n + 31) >> 5;
             pu_batch = 0;
@@ -444,9 +490,27 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
 
     for (int i = 0; i < stages && !pu_done; ++i) produce();
 
+    // Publishes a stored partial: fence, ticket, and the merge if this was the last split to arrive.
+    PendingArrival pend{0, 0, 0, 0, 0, 0};
+    auto publish = [&]() {
+        if (!pend.valid) return;
+        pend.valid = 0;
+        __threadfence();
+        __syncwarp();
+        int ticket = 0;
+        if (lane == 0) ticket = atomicAdd(&p.tickets[pend.ticket_idx], 1);
+        ticket = __shfl_sync(kFull, ticket, 0);
+        if (ticket == pend.nc - 1) {
+            if (lane == 0) p.tickets[pend.ticket_idx] = 0;   // ready for the next launch
+            __threadfence();
+            for (int g = 0; g < GT; ++g)
+                merge_partials_row<D, BF16>(p, pend.wf, pend.wf_slot, pend.nc, g, GT, pend.row0 + g, lane);
+        }
+    };
+
     // ---- consumer
-    float q[GT][E], o[GT][E], m[GT], l[GT];
-    int cur_unit = -1;
+    float q[GT][E], o[GT][E], m[GT], l[GT], sc[BT / 4][GT];
+    int cur_seg = -1;
     int cons_stage = 0;
     uint32_t cons_phase = 0;
     while (inflight > 0) {
@@ -462,11 +526,12 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
             return;
         }
         const int32_t *mt = meta + cons_stage * M_WORDS;
-        const int unit = mt[M_UNIT], s = mt[M_SEQ], hg = mt[M_HG], c = mt[M_C], nu = mt[M_NU];
-        const int ntok = mt[M_NTOK];
-        const bool last = mt[M_LAST] != 0;
-        if (unit != cur_unit) {
-            cur_unit = unit;
+        const int seg = mt[M_SEG], s = mt[M_SEQ], hg = mt[M_HG], nc = mt[M_NC];
+        const int ntok = mt[M_NTOK], flags = mt[M_FLAGS];
+        const int mt_wf = mt[M_WF], mt_wfslot = mt[M_WFSLOT];
+        const int kind = flags & F_KIND_MASK;
+        if (seg != cur_seg) {
+            cur_seg = seg;
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
                 const uint16_t *qrow =
@@ -485,9 +550,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
                 for (int e = 0; e < E; ++e) o[g][e] = 0.f;
             }
         }
-        if (ntok > 0) {
-            const uint8_t *sK = data + (size_t)cons_stage * STAGE;
-            tile_compute<D, GT, BT, BF16>(sK, sK + TILE, ntok, grp, sub, q, o, m, l);
+        const uint8_t *tile = data + (size_t)cons_stage * TILE;
+        if (kind == F_KIND_K) {
+            tile_scores<D, GT, BT, BF16>(tile, ntok, grp, sub, q, sc, o, m, l);
+        } else if (kind == F_KIND_V) {
+            tile_values<D, GT, BT, BF16>(tile, ntok, grp, sub, sc, o, m, l);
         }
         __syncwarp();   // every lane is done with this stage (data and metadata) before it is refilled
         --inflight;
@@ -495,7 +562,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
         if (cons_stage == 0) cons_phase ^= 1u;
         if (!pu_done) produce();
 
-        if (!last) continue;
+        if (!(flags & F_LAST)) continue;
 
         // ---- end of unit: merge the four token groups of the warp
 #pragma unroll
@@ -548,7 +615,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
         }
 
         // ---- resident mode
-        if (nu == 1) {   // the unit covered the whole sequence: no partial needed
+        if (nc == 1) {   // this warp covered the whole (sequence, head group): no partial needed
             if (grp == 0) {
 #pragma unroll
                 for (int g = 0; g < GT; ++g) {
@@ -566,10 +633,12 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
             }
             continue;
         }
+        publish();   // the previous partial's arrival; its stores have long landed
+        const int slot = 2 * gw + (seg == 0 ? 0 : 1);   // an incomplete segment is the warp's first or its last
         if (grp == 0) {
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
-                const size_t pr = (size_t)unit * GT + g;
+                const size_t pr = (size_t)slot * GT + g;
                 store_row_grouped<D, BF16>(nullptr, p.part_o, pr, sub, o[g], 1.f);
                 if (sub == 0) {
                     p.part_ml[pr * 2] = m[g];
@@ -577,19 +646,14 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, 1) decode_kernel(const Deco
                 }
             }
         }
-        __threadfence();
-        __syncwarp();
-        int ticket = 0;
-        if (lane == 0) ticket = atomicAdd(&p.tickets[s * Hg + hg], 1);
-        ticket = __shfl_sync(kFull, ticket, 0);
-        if (ticket == nu - 1) {
-            if (lane == 0) p.tickets[s * Hg + hg] = 0;   // ready for the next launch
-            __threadfence();
-            const int u0 = unit - c;
-            for (int g = 0; g < GT; ++g)
-                merge_partials_row<D, BF16>(p, u0, nu, g, GT, (size_t)s * p.Hq + (size_t)hg * GT + g, lane);
-        }
+        pend.valid = 1;
+        pend.ticket_idx = s * Hg + hg;
+        pend.nc = nc;
+        pend.wf = mt_wf;
+        pend.wf_slot = mt_wfslot;
+        pend.row0 = (size_t)s * p.Hq + (size_t)hg * GT;
     }
+    publish();
 }
 
 // ---------------------------------------------------------------- merge kernel (resident + offloaded)
@@ -742,12 +806,17 @@ __global__ void gather_kernel(const GatherParams p) {
 
 // ---------------------------------------------------------------- dispatch
 
+#ifndef ISV_WARPS_GT1
+#define ISV_WARPS_GT1 16   // warps per CTA when one query head is handled per KV tile
+#endif
+
 typedef void (*DecodeFn)(const DecodeParams, const int);
 
 template <int D, int GT, bool BF16>
 DecodeFn pick_mode(int mode) {
-    return mode == MODE_RESIDENT ? decode_kernel<D, GT, 16, BF16, MODE_RESIDENT>
-                                 : decode_kernel<D, GT, 16, BF16, MODE_STAGED>;
+    constexpr int NW = GT == 1 ? ISV_WARPS_GT1 : 8;
+    return mode == MODE_RESIDENT ? decode_kernel<D, GT, 16, BF16, MODE_RESIDENT, NW>
+                                 : decode_kernel<D, GT, 16, BF16, MODE_STAGED, NW>;
 }
 template <int D, int GT>
 DecodeFn pick_dtype(bool bf16, int mode) {
@@ -771,9 +840,11 @@ DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
 
 }  // namespace
 
-size_t decode_smem_bytes(int D, int BT, int stages, int max_seqs, int mode) {
-    const size_t stage = 2ull * BT * D * 2;
-    size_t b = (size_t)kDecodeWarps * stages * (stage + 8 + 4 * M_WORDS);
+int decode_warps(int GT) { return GT == 1 ? ISV_WARPS_GT1 : 8; }
+
+size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode) {
+    const size_t tile = (size_t)BT * D * 2;
+    size_t b = (size_t)decode_warps(GT) * stages * (tile + 8 + 4 * M_WORDS);
     if (mode == MODE_RESIDENT) b += (size_t)(max_seqs + 1) * 4;
     return b;
 }
@@ -788,7 +859,7 @@ cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int BT, bool bf1
                           int stages, size_t smem, cudaStream_t st) {
     DecodeFn fn = pick(D, GT, BT, bf16, mode);
     if (!fn) return cudaErrorInvalidValue;
-    fn<<<grid, kDecodeWarps * 32, smem, st>>>(p, stages);
+    fn<<<grid, decode_warps(GT) * 32, smem, st>>>(p, stages);
     return cudaGetLastError();
 }
 

@@ -7,17 +7,17 @@
 
 namespace isv {
 
-constexpr int kDecodeWarps = 8;          // consumer warps per CTA of the decode kernel
 constexpr int kMaxTableUpdates = 480;    // entries one update launch carries by value
 
 enum DecodeMode : int { MODE_RESIDENT = 0, MODE_STAGED = 1 };
 
 // One launch of the split decode kernel.
-//   MODE_RESIDENT: units are (sequence, kv head x pass, split of `U` logical
-//     blocks); the kernel walks the block table, reads HBM-pool blocks and a
+//   MODE_RESIDENT: the KV blocks of all (sequence, kv head x pass) pairs form
+//     one flat list that is cut into equal contiguous ranges, one per warp; a
+//     warp walks the block table for its range, reads HBM-pool blocks and a
 //     host-flagged newest block from its tail slot, skips other host blocks.
-//     Each (sequence, head group) is finished by whichever unit arrives last
-//     (ticket), which merges the splits' partials.
+//     A (sequence, head group) that spans several warps is finished by
+//     whichever of them arrives last (ticket), which merges their partials.
 //   MODE_STAGED: units are (chunk unit, kv head x pass) from the plan lists;
 //     blocks are read from the staging buffer; results are merged into the
 //     running state acc_o / acc_ml, which one unit per launch owns.
@@ -40,13 +40,13 @@ struct DecodeParams {
     void *out;                  // [n_seqs][Hq][D] 16-bit or NULL
     float *out_f32;             // [n_seqs][Hq][D] or NULL
     // scratch
-    float *part_o;              // [units][GT][D]
-    float *part_ml;             // [units][GT][2]
+    float *part_o;              // [2 * warps in grid][GT][D]   (a warp leaves at most two partials)
+    float *part_ml;             // [2 * warps in grid][GT][2]
     int32_t *tickets;           // [n_seqs][Hkv*P], zero between launches
     float *acc_o;               // [n_seqs][Hq][D]  unnormalised result (resident, !finalize) / running state (staged)
     float *acc_ml;              // [n_seqs][Hq][2]
     uint32_t *status;
-    int32_t n_seqs, Hq, Hkv, P, U;
+    int32_t n_seqs, Hq, Hkv, P;
     int32_t finalize;           // resident: 1 = normalise and write out; 0 = leave (m, l, o) in acc_*
     float scale_log2;           // log2(e) / sqrt(D)
     uint64_t block_bytes;
@@ -99,9 +99,12 @@ struct MergeParams {
     int32_t rows, D, bf16;
 };
 
+// Warps per CTA of the decode kernel that handles GT query heads per KV tile.
+int decode_warps(int GT);
+
 // Bytes of dynamic shared memory the decode kernel needs for `stages` ring
-// stages per warp.
-size_t decode_smem_bytes(int D, int BT, int stages, int max_seqs, int mode);
+// stages (one K or V tile each) per warp.
+size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode);
 
 // Launchers return the CUDA error of the launch.
 cudaError_t decode_configure(int D, int GT, int BT, bool bf16, int mode, size_t smem);

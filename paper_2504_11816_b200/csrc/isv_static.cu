@@ -64,7 +64,7 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
                                       const int32_t *block_table_dev, int32_t table_stride,
                                       const int32_t *seq_lens_dev, int32_t n_seqs, int32_t max_blocks_per_seq,
                                       int32_t q_heads, int32_t kv_heads, int32_t head_dim, int32_t block_tokens,
-                                      int32_t dtype, int32_t split_blocks, const void *q_dev, void *out_dev,
+                                      int32_t dtype, int32_t max_ctas, const void *q_dev, void *out_dev,
                                       float *out_f32_dev, uint32_t *status_dev, void *stream) {
     if (!kv_pool_dev || !block_table_dev || !seq_lens_dev || !q_dev || (!out_dev && !out_f32_dev))
         return err(ISV_EINVAL, "isv_attn_decode_static: pool, table, lengths, q and one output are required");
@@ -76,7 +76,7 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     if ((head_dim != 64 && head_dim != 128) || block_tokens != 16 || (dtype != ISV_F16 && dtype != ISV_BF16))
         return err(ISV_EINVAL, "isv_attn_decode_static: head_dim 64/128, block_tokens 16, dtype f16/bf16 only");
     if (n_seqs < 0 || n_seqs > 4096 || max_blocks_per_seq < 1 || table_stride < max_blocks_per_seq ||
-        n_pool_blocks < 1 || split_blocks < 0)
+        n_pool_blocks < 1 || max_ctas < 0)
         return err(ISV_EINVAL, "isv_attn_decode_static: bad n_seqs (%d) or block counts (%d)", n_seqs,
                    max_blocks_per_seq);
     if (n_seqs == 0) return ISV_OK;
@@ -84,19 +84,8 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     const int G = q_heads / kv_heads;
     const int GT = (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
     const int P = G / GT;
-    const int U = split_blocks == 0 ? 8 : split_blocks;
-    const size_t rows = (size_t)n_seqs * q_heads;
-    const size_t splits = ((size_t)max_blocks_per_seq + U - 1) / U;
-    const size_t tickets_bytes = align256((size_t)n_seqs * kv_heads * P * 4);
-    const size_t ml_bytes = align256(rows * splits * 2 * 4);
-    const size_t o_bytes = rows * splits * head_dim * 4;
-    const size_t need = kHeaderBytes + tickets_bytes + ml_bytes + o_bytes;
-    if (need > (size_t)ISV_STATIC_SCRATCH_BYTES)
-        return err(ISV_ECAPACITY,
-                   "isv_attn_decode_static: this shape needs %lld bytes of split scratch but the fixed array holds "
-                   "%lld; use fewer sequences, shorter sequences or a larger split_blocks, or the handle-based "
-                   "isv_attn_decode",
-                   (long long)need, (long long)ISV_STATIC_SCRATCH_BYTES);
+    if ((long long)n_seqs * max_blocks_per_seq * kv_heads * P >= (1ll << 31))
+        return err(ISV_EINVAL, "isv_attn_decode_static: n_seqs * blocks * heads too large");
 
     // ---- once per device: address of the scratch symbol and device limits
     int dev = 0;
@@ -125,12 +114,29 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
         ds = g_dev[dev];
     }
 
+    // ---- scratch: counters per (sequence, head group) and two partials per warp of the grid
+    const int nw = decode_warps(GT);
+    const long long blocks = (long long)n_seqs * max_blocks_per_seq * kv_heads * P;
+    const int cap = max_ctas > 0 ? std::min(max_ctas, ds.sm_count) : ds.sm_count;
+    const int grid = (int)std::max<long long>(1, std::min<long long>(cap, (blocks + nw - 1) / nw));
+    const size_t slots = 2ull * grid * nw * GT;
+    const size_t tickets_bytes = align256((size_t)n_seqs * kv_heads * P * 4);
+    const size_t ml_bytes = align256(slots * 2 * 4);
+    const size_t o_bytes = slots * head_dim * 4;
+    const size_t need = kHeaderBytes + tickets_bytes + ml_bytes + o_bytes;
+    if (need > (size_t)ISV_STATIC_SCRATCH_BYTES)
+        return err(ISV_ECAPACITY,
+                   "isv_attn_decode_static: this shape needs %lld bytes of scratch (arrival counters for %d sequences "
+                   "x %d head groups plus split partials) but the fixed array holds %lld; use fewer sequences or "
+                   "heads per call, a smaller max_ctas, or the handle-based isv_attn_decode",
+                   (long long)need, n_seqs, kv_heads * P, (long long)ISV_STATIC_SCRATCH_BYTES);
+
     // ---- shared-memory ring depth that fits
     const bool bf16 = dtype == ISV_BF16;
     int stages = 0;
     size_t smem = 0;
-    for (int st = 2; st <= 8; ++st) {
-        const size_t b = decode_smem_bytes(head_dim, block_tokens, st, n_seqs, MODE_RESIDENT);
+    for (int st = 2; st <= 12; ++st) {
+        const size_t b = decode_smem_bytes(head_dim, block_tokens, GT, st, n_seqs, MODE_RESIDENT);
         if (b <= (size_t)ds.smem_optin) { stages = st; smem = b; }
     }
     if (stages < 2) return err(ISV_EINVAL, "isv_attn_decode_static: shared memory too small for this shape");
@@ -160,13 +166,10 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     p.part_o = reinterpret_cast<float *>(base + kHeaderBytes + tickets_bytes + ml_bytes);
     p.acc_o = nullptr;
     p.acc_ml = nullptr;
-    p.n_seqs = n_seqs; p.Hq = q_heads; p.Hkv = kv_heads; p.P = P; p.U = U;
+    p.n_seqs = n_seqs; p.Hq = q_heads; p.Hkv = kv_heads; p.P = P;
     p.finalize = 1;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)head_dim));
     p.block_bytes = 2ull * kv_heads * block_tokens * head_dim * 2ull;
-    // the kernel is persistent: one CTA per SM covers any number of units
-    const long long max_units = (long long)n_seqs * kv_heads * P * (long long)splits;
-    const int grid = (int)std::max<long long>(1, std::min<long long>(ds.sm_count, (max_units + kDecodeWarps - 1) / kDecodeWarps));
     e = launch_decode(p, head_dim, GT, block_tokens, bf16, MODE_RESIDENT, grid, stages, smem, st);
     if (e != cudaSuccess) return err(ISV_ECUDA, "isv_attn_decode_static: %s", cudaGetErrorString(e));
     return ISV_OK;

@@ -40,7 +40,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_bad_descriptions_are_rejected_with_a_message():
     for kw in (dict(head_dim=96), dict(q_heads=6, kv_heads=4), dict(offload_frac=1.5), dict(block_tokens=8),
-               dict(max_seqs=0), dict(layers=0), dict(phys_layers=3), dict(dtype=7), dict(ring_depth=1)):
+               dict(max_seqs=0), dict(layers=0), dict(phys_layers=3), dict(dtype=7), dict(ring_depth=1), dict(max_ctas=-1)):
         with pytest.raises(B.IsvError) as ei:
             _alloc(**kw)
         assert ei.value.code == B.ISV_EINVAL and ei.value.message

@@ -88,8 +88,8 @@ def test_static_entry_matches_handle_entry_on_two_calls_in_a_row(q_heads, kv_hea
 def test_static_entry_refuses_shapes_beyond_its_fixed_scratch():
     one = torch.zeros(64, dtype=torch.int32, device="cuda")
     with pytest.raises(B.IsvError) as ei:
-        # 256 sequences x 32 heads x 4096 tokens: far more split scratch than the fixed array holds
-        B.isv_attn_decode_static(one, 1, one, 256, one, 256, 256, 32, 32, 128, 16, B.ISV_F16, 0, one, one, None,
+        # 4096 sequences x 256 head groups: the arrival counters plus the partials exceed the fixed array
+        B.isv_attn_decode_static(one, 1, one, 64, one, 4096, 64, 1024, 256, 128, 16, B.ISV_F16, 0, one, one, None,
                                  None, 0)
     assert ei.value.code == B.ISV_ECAPACITY
     assert "fixed array" in ei.value.message
