@@ -123,7 +123,7 @@ typedef struct {
  * bytes_staged is what the copy engine actually moved (whole chunks).
  */
 typedef struct {
-    float    append_ms;
+    float    append_ms;           /* 0 when the append was fused into the attention kernel */
     float    h2d_ms;
     float    attn_resident_ms;
     float    attn_offloaded_ms;
@@ -186,7 +186,15 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q_dev, void *out_dev,
                     float *out_f32_dev, const int32_t *block_table_dev,
                     const int32_t *seq_lens_dev, int32_t n_seqs);
 
-/* One decode step of all layers: for l in 0..layers-1 append then attend.
+/* isv_kv_append followed by isv_attn_decode for one layer, as one kernel: the
+ * resident attention kernel also stores the new token's K/V rows and advances
+ * the lengths, and attends to the new token straight from k_dev / v_dev, so
+ * the step needs one launch per layer instead of two.  Same arguments and
+ * result as the two calls (up to fp32 summation order). */
+int isv_decode_layer(isv_kv *h, int32_t layer, const void *q_dev, const void *k_dev, const void *v_dev,
+                     void *out_dev, float *out_f32_dev, int32_t n_seqs);
+
+/* One decode step of all layers: isv_decode_layer for l in 0..layers-1.
  * Device arrays: q, out [layers][n_seqs][q_heads][head_dim];
  * k, v [layers][n_seqs][kv_heads][head_dim]. */
 int isv_decode_step(isv_kv *h, const void *q_dev, const void *k_dev, const void *v_dev,

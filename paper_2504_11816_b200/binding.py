@@ -33,7 +33,7 @@ ISV_BLOCK_HOST_BIT = 1 << 30
 
 EXPORTS = [
     "isv_kv_alloc", "isv_kv_free", "isv_kv_reset", "isv_kv_info", "isv_kv_fill", "isv_kv_append",
-    "isv_attn_decode", "isv_decode_step", "isv_decode_step_host", "isv_kv_gather",
+    "isv_attn_decode", "isv_decode_layer", "isv_decode_step", "isv_decode_step_host", "isv_kv_gather",
     "isv_block_table_dev", "isv_seq_lens_dev", "isv_block_table_host", "isv_seq_lens_host",
     "isv_plan_bytes", "isv_set_timing", "isv_step_timing", "isv_sync", "isv_link_probe",
     "isv_attn_decode_static", "isv_last_error",
@@ -109,6 +109,7 @@ def lib():
     L.isv_kv_fill.argtypes = [vp, i32, vp, vp, vp, i32, i32]
     L.isv_kv_append.argtypes = [vp, i32, vp, vp, i32]
     L.isv_attn_decode.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32]
+    L.isv_decode_layer.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32]
     L.isv_decode_step.argtypes = [vp, vp, vp, vp, vp, i32]
     L.isv_decode_step_host.argtypes = [vp, vp, vp, vp, vp, i32]
     L.isv_kv_gather.argtypes = [vp, i32, i32, vp, vp, P(i32)]
@@ -196,6 +197,10 @@ def isv_kv_append(h: int, layer: int, k, v, n_seqs: int):
 def isv_attn_decode(h: int, layer: int, q, out, out_f32, block_table, seq_lens, n_seqs: int):
     _check(lib().isv_attn_decode(h, layer, _ptr(q), _ptr(out), _ptr(out_f32), _ptr(block_table),
                                  _ptr(seq_lens), n_seqs))
+
+
+def isv_decode_layer(h: int, layer: int, q, k, v, out, out_f32, n_seqs: int):
+    _check(lib().isv_decode_layer(h, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(out_f32), n_seqs))
 
 
 def isv_decode_step(h: int, q, k, v, out, n_seqs: int):

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -51,7 +52,7 @@ struct PlanSlot {
 
 struct LayerEvents {
     cudaEvent_t a0, a1, d0, d1, r0, r1, c0, c1, o0, o1, m0, m1;
-    bool have_append = false, have_decode = false, have_off = false;
+    bool have_append = false, have_decode = false, have_off = false, fused_append = false;
     uint64_t bytes_res = 0, bytes_off = 0, bytes_staged = 0, bytes_app = 0;
     int n_chunks = 0;
 };
@@ -66,7 +67,8 @@ struct isv_kv {
     // device memory
     uint8_t *pool_hbm = nullptr, *tail = nullptr;
     uint8_t *pool_host = nullptr, *pool_host_dev = nullptr;   // pinned host pool and its device alias
-    int32_t *table_dev = nullptr, *lens_dev = nullptr;
+    int32_t *table_dev = nullptr, *lens_dev = nullptr;   // lens_dev: two copies of [layers][max_seqs]
+    std::vector<char> lens_cur;            // per layer: which copy is current
     uint32_t *status_dev = nullptr;
     float *part_o = nullptr, *part_ml = nullptr, *res_o = nullptr, *res_ml = nullptr, *run_o = nullptr,
           *run_ml = nullptr;
@@ -96,6 +98,13 @@ struct isv_kv {
 };
 
 namespace {
+
+// Device lengths of one layer: the current copy (which = 0) or the other one (which = 1).  The fused
+// append + attention kernel reads the current copy and writes the other, then they swap.
+int32_t *lens_ptr(const isv_kv *h, int layer, int which) {
+    const int copy = (h->lens_cur[layer] ^ which) & 1;
+    return h->lens_dev + ((size_t)copy * h->g.layers + layer) * h->g.max_seqs;
+}
 
 size_t slab_hbm(const isv_kv *h, int layer) {
     return (size_t)(layer % h->g.phys_layers) * h->g.hbm_cap * h->g.block_bytes;
@@ -155,9 +164,12 @@ int dev_alloc(void **p, size_t bytes, uint64_t *tally, const char *what) {
     return ISV_OK;
 }
 
+// Ring depth per warp: the default depth (or ISV_DECODE_STAGES, a tuning knob), reduced until it fits.
 int pick_stages(const Geometry &g, int mode, int smem_limit, size_t *smem_out) {
     int best = 0;
-    for (int st = 2; st <= 12; ++st) {
+    int cap = decode_default_stages(g.D, g.BT, g.GT);
+    if (const char *e = getenv("ISV_DECODE_STAGES")) cap = std::max(2, std::min(12, atoi(e)));
+    for (int st = 2; st <= cap; ++st) {
         const size_t b = decode_smem_bytes(g.D, g.BT, g.GT, st, g.max_seqs, mode);
         if (b <= (size_t)smem_limit) { best = st; *smem_out = b; }
     }
@@ -262,6 +274,36 @@ int upload_plan(isv_kv *h, const OffPlan &pl, PlanSlot **out) {
     return ISV_OK;
 }
 
+struct AppendPlan {
+    std::vector<TableUpdate> upd;   // table entries of blocks allocated for this step
+    std::vector<int> flush;         // sequences whose host-flagged newest block becomes full
+    bool new_host_block = false;    // some sequence starts a host-flagged block (needs its tail slot free)
+};
+
+// Host side of appending one token to sequences [0, n_seqs) of a layer: capacity checks, block
+// allocation by the residency rule, length mirror.  Nothing is changed when an error is returned.
+int append_bookkeeping(isv_kv *h, int layer, int n_seqs, AppendPlan *ap) {
+    const Geometry &g = h->g;
+    if (n_seqs < 0 || n_seqs > g.max_seqs) return fail(ISV_EINVAL, "n_seqs %d outside [0, %d]", n_seqs, g.max_seqs);
+    std::vector<std::pair<int, int>> need;
+    for (int s = 0; s < n_seqs; ++s) {
+        const int pos = h->bm.length(layer, s);
+        if (pos >= g.max_tokens) return fail(ISV_ECAPACITY, "sequence %d is full (%d tokens)", s, pos);
+        if (pos % g.BT == 0) {
+            const int j = pos / g.BT;
+            if (h->bm.entry(s, j) == ISV_BLOCK_NONE) need.push_back({s, j});
+            if (h->bm.is_host(j)) ap->new_host_block = true;
+        }
+    }
+    int rc = h->bm.allocate(need, &ap->upd);
+    if (rc) return fail(rc, "KV pool full");
+    for (int s = 0; s < n_seqs; ++s) {
+        const int n = ++h->bm.length(layer, s);
+        if (n % g.BT == 0 && h->bm.is_host((n - 1) / g.BT)) ap->flush.push_back(s);
+    }
+    return ISV_OK;
+}
+
 }  // namespace
 
 // Lets the library's other translation units record the calling thread's last error.
@@ -343,10 +385,11 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
     }
     // tables
     if ((rc = dev_alloc((void **)&h->table_dev, (size_t)g.max_seqs * g.NB * 4, nullptr, "block table"))) return bail(rc);
-    if ((rc = dev_alloc((void **)&h->lens_dev, (size_t)g.layers * g.max_seqs * 4, nullptr, "lengths"))) return bail(rc);
+    if ((rc = dev_alloc((void **)&h->lens_dev, 2 * (size_t)g.layers * g.max_seqs * 4, nullptr, "lengths"))) return bail(rc);
+    h->lens_cur.assign(g.layers, 0);
     if ((rc = dev_alloc((void **)&h->status_dev, 4, nullptr, "status"))) return bail(rc);
     CUB(cudaMemset(h->table_dev, 0xff, (size_t)g.max_seqs * g.NB * 4));
-    CUB(cudaMemset(h->lens_dev, 0, (size_t)g.layers * g.max_seqs * 4));
+    CUB(cudaMemset(h->lens_dev, 0, 2 * (size_t)g.layers * g.max_seqs * 4));
     CUB(cudaMemset(h->status_dev, 0, 4));
     // scratch
     const size_t rows = (size_t)g.max_seqs * g.Hq;
@@ -415,7 +458,7 @@ int isv_kv_reset(isv_kv *h) {
         int rc = isv_sync(h, nullptr);
         if (rc && rc != ISV_EDEVICE_STATUS) return rc;
         CU(cudaMemset(h->table_dev, 0xff, (size_t)h->g.max_seqs * h->g.NB * 4));
-        CU(cudaMemset(h->lens_dev, 0, (size_t)h->g.layers * h->g.max_seqs * 4));
+        CU(cudaMemset(h->lens_dev, 0, 2 * (size_t)h->g.layers * h->g.max_seqs * 4));
         CU(cudaMemset(h->tickets, 0, (size_t)h->g.max_seqs * h->g.Hkv * h->g.P * 4));
         std::fill(h->flush_recorded.begin(), h->flush_recorded.end(), 0);
     }
@@ -468,7 +511,7 @@ int isv_kv_fill(isv_kv *h, int32_t layer, const void *k, const void *v, const in
 
     CU(cudaStreamSynchronize(h->s_compute));
     CU(cudaMemcpy(h->table_dev, h->bm.table.data(), h->bm.table.size() * 4, cudaMemcpyHostToDevice));
-    CU(cudaMemcpy(h->lens_dev + (size_t)layer * g.max_seqs, &h->bm.len[(size_t)layer * g.max_seqs],
+    CU(cudaMemcpy(lens_ptr(h, layer, 0), &h->bm.len[(size_t)layer * g.max_seqs],
                   (size_t)g.max_seqs * 4, cudaMemcpyHostToDevice));
     const int pl = layer % g.phys_layers;
     if (h->flush_recorded[pl]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_flush[pl], 0));
@@ -481,7 +524,7 @@ int isv_kv_fill(isv_kv *h, int32_t layer, const void *k, const void *v, const in
         p.tail = h->tail ? h->tail + slab_tail(h, layer) : nullptr;
         p.host = h->pool_host_dev ? h->pool_host_dev + slab_host(h, layer) : nullptr;
         p.table = h->table_dev;
-        p.lens = h->lens_dev + (size_t)layer * g.max_seqs;
+        p.lens = lens_ptr(h, layer, 0);
         p.status = h->status_dev;
         p.table_stride = g.NB; p.n_pool_blocks = g.hbm_cap; p.n_host_blocks = g.host_cap;
         p.n_seqs = n_seqs; p.T = T; p.Hkv = g.Hkv; p.D = g.D; p.BT = g.BT; p.max_blocks = max_blocks;
@@ -505,45 +548,27 @@ int isv_kv_append(isv_kv *h, int32_t layer, const void *k, const void *v, int32_
     int rc = check_handle(h, layer, false);
     if (rc) return rc;
     const Geometry &g = h->g;
-    if (n_seqs < 0 || n_seqs > g.max_seqs) return fail(ISV_EINVAL, "n_seqs %d outside [0, %d]", n_seqs, g.max_seqs);
     if (!h->plan_only && (!k || !v || !aligned16(k) || !aligned16(v)))
         return fail(ISV_EINVAL, "k and v must be non-null and 16-byte aligned");
-    if (n_seqs == 0) return ISV_OK;
-    std::vector<std::pair<int, int>> need;
-    bool new_host_block = false;
-    for (int s = 0; s < n_seqs; ++s) {
-        const int pos = h->bm.length(layer, s);
-        if (pos >= g.max_tokens) return fail(ISV_ECAPACITY, "sequence %d is full (%d tokens)", s, pos);
-        if (pos % g.BT == 0) {
-            const int j = pos / g.BT;
-            if (h->bm.entry(s, j) == ISV_BLOCK_NONE) need.push_back({s, j});
-            if (h->bm.is_host(j)) new_host_block = true;
-        }
-    }
-    std::vector<TableUpdate> upd;
-    if ((rc = h->bm.allocate(need, &upd))) return fail(rc, "KV pool full");
-    std::vector<int> flush;
-    for (int s = 0; s < n_seqs; ++s) {
-        const int n = ++h->bm.length(layer, s);
-        if (n % g.BT == 0 && h->bm.is_host((n - 1) / g.BT)) flush.push_back(s);
-    }
-    if (h->plan_only) return ISV_OK;
+    AppendPlan ap;
+    if ((rc = append_bookkeeping(h, layer, n_seqs, &ap))) return rc;
+    if (h->plan_only || n_seqs == 0) return ISV_OK;
 
     LayerEvents *le = nullptr;
     if (h->timing) {
         le = &h->lev[layer];
         CU(cudaEventRecord(le->a0, h->s_compute));
     }
-    if ((rc = push_updates(h, upd))) return rc;
+    if ((rc = push_updates(h, ap.upd))) return rc;
     const int pl = layer % g.phys_layers;
     // a tail slot about to take a new block must have finished its write-back
-    if (new_host_block && h->flush_recorded[pl]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_flush[pl], 0));
+    if (ap.new_host_block && h->flush_recorded[pl]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_flush[pl], 0));
     AppendParams p{};
     p.k = k; p.v = v;
     p.pool = h->pool_hbm + slab_hbm(h, layer);
     p.tail = h->tail ? h->tail + slab_tail(h, layer) : nullptr;
     p.table = h->table_dev;
-    p.lens = h->lens_dev + (size_t)layer * g.max_seqs;
+    p.lens = lens_ptr(h, layer, 0);
     p.status = h->status_dev;
     p.table_stride = g.NB; p.n_pool_blocks = g.hbm_cap;
     p.n_seqs = n_seqs; p.Hkv = g.Hkv; p.D = g.D; p.BT = g.BT;
@@ -553,15 +578,18 @@ int isv_kv_append(isv_kv *h, int32_t layer, const void *k, const void *v, int32_
     if (le) {
         CU(cudaEventRecord(le->a1, h->s_compute));
         le->have_append = true;
+        le->fused_append = false;
         le->bytes_app = (uint64_t)n_seqs * g.kappa;
     }
-    return flush_tails(h, layer, flush);
+    return flush_tails(h, layer, ap.flush);
 }
 
-int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *out_f32,
-                    const int32_t *block_table_dev, const int32_t *seq_lens_dev, int32_t n_seqs) {
-    int rc = check_handle(h, layer, true);
-    if (rc) return rc;
+// Attention of one layer; with k_new / v_new also this step's append, fused into the resident kernel
+// (the device lengths then still hold the values before the append and the kernel advances them).
+static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float *out_f32,
+                       const int32_t *block_table_dev, const int32_t *seq_lens_dev, int32_t n_seqs,
+                       const void *k_new, const void *v_new) {
+    int rc = ISV_OK;
     const Geometry &g = h->g;
     if (n_seqs < 0 || n_seqs > g.max_seqs) return fail(ISV_EINVAL, "n_seqs %d outside [0, %d]", n_seqs, g.max_seqs);
     if (!q || (!out && !out_f32)) return fail(ISV_EINVAL, "q and one of out / out_f32 must be given");
@@ -589,7 +617,7 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *o
 
     DecodeParams base{};
     base.table = block_table_dev ? block_table_dev : h->table_dev;
-    base.lens = seq_lens_dev ? seq_lens_dev : h->lens_dev + (size_t)layer * g.max_seqs;
+    base.lens = seq_lens_dev ? seq_lens_dev : lens_ptr(h, layer, 0);
     base.table_stride = g.NB;
     base.q = q;
     base.status = h->status_dev;
@@ -655,6 +683,12 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *o
         p.part_o = h->part_o; p.part_ml = h->part_ml; p.tickets = h->tickets;
         p.acc_o = h->res_o; p.acc_ml = h->res_ml;
         p.finalize = offloaded ? 0 : 1;
+        if (k_new) {
+            p.k_new = k_new; p.v_new = v_new;
+            p.lens_out = lens_ptr(h, layer, 1);
+            p.pool_w = h->pool_hbm + slab_hbm(h, layer);
+            p.tail_w = h->tail ? h->tail + slab_tail(h, layer) : nullptr;
+        }
         long long nu = 0;   // KV blocks in the flat work list
         for (int s = 0; s < n_seqs; ++s)
             nu += (long long)std::max(1, (h->bm.length(layer, s) + g.BT - 1) / g.BT) * Hg;
@@ -664,6 +698,7 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *o
         CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_RESIDENT, grid, h->stages_res, h->smem_res, h->s_compute));
         ++h->launches;
         if (le) CU(cudaEventRecord(le->r1, h->s_compute));
+        if (k_new) h->lens_cur[layer] ^= 1;   // the kernel wrote the advanced lengths to the other copy
     }
 
     if (offloaded) {
@@ -681,6 +716,36 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *o
     return ISV_OK;
 }
 
+int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *out_f32,
+                    const int32_t *block_table_dev, const int32_t *seq_lens_dev, int32_t n_seqs) {
+    int rc = check_handle(h, layer, true);
+    if (rc) return rc;
+    return decode_impl(h, layer, q, out, out_f32, block_table_dev, seq_lens_dev, n_seqs, nullptr, nullptr);
+}
+
+int isv_decode_layer(isv_kv *h, int32_t layer, const void *q, const void *k, const void *v, void *out,
+                     float *out_f32, int32_t n_seqs) {
+    int rc = check_handle(h, layer, true);
+    if (rc) return rc;
+    const Geometry &g = h->g;
+    if (!k || !v || !aligned16(k) || !aligned16(v)) return fail(ISV_EINVAL, "k and v must be non-null and 16-byte aligned");
+    if (!q || (!out && !out_f32) || !aligned16(q) || !aligned16(out) || !aligned16(out_f32))
+        return fail(ISV_EINVAL, "q and one of out / out_f32 must be given, 16-byte aligned");
+    AppendPlan ap;
+    if ((rc = append_bookkeeping(h, layer, n_seqs, &ap))) return rc;
+    if (n_seqs == 0) return ISV_OK;
+    if (h->timing) {
+        h->lev[layer].have_append = false;
+        h->lev[layer].fused_append = true;
+    }
+    if ((rc = push_updates(h, ap.upd))) return rc;
+    const int pl = layer % g.phys_layers;
+    if (ap.new_host_block && h->flush_recorded[pl]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_flush[pl], 0));
+    if ((rc = decode_impl(h, layer, q, out, out_f32, nullptr, nullptr, n_seqs, k, v))) return rc;
+    if (h->timing) h->lev[layer].bytes_app = (uint64_t)n_seqs * g.kappa;
+    return flush_tails(h, layer, ap.flush);
+}
+
 int isv_decode_step(isv_kv *h, const void *q, const void *k, const void *v, void *out, int32_t n_seqs) {
     int rc = check_handle(h, 0, true);
     if (rc) return rc;
@@ -689,8 +754,8 @@ int isv_decode_step(isv_kv *h, const void *q, const void *k, const void *v, void
     if (n_seqs < 0 || n_seqs > g.max_seqs) return fail(ISV_EINVAL, "n_seqs %d outside [0, %d]", n_seqs, g.max_seqs);
     const size_t qs = (size_t)n_seqs * g.Hq * g.D * 2, ks = (size_t)n_seqs * g.Hkv * g.D * 2;
     for (int l = 0; l < g.layers; ++l) {
-        if ((rc = isv_kv_append(h, l, (const uint8_t *)k + l * ks, (const uint8_t *)v + l * ks, n_seqs))) return rc;
-        if ((rc = isv_attn_decode(h, l, (const uint8_t *)q + l * qs, (uint8_t *)out + l * qs, nullptr, nullptr, nullptr, n_seqs)))
+        if ((rc = isv_decode_layer(h, l, (const uint8_t *)q + l * qs, (const uint8_t *)k + l * ks,
+                                   (const uint8_t *)v + l * ks, (uint8_t *)out + l * qs, nullptr, n_seqs)))
             return rc;
     }
     return ISV_OK;
@@ -757,7 +822,7 @@ const int32_t *isv_block_table_dev(isv_kv *h, int32_t *row_stride) {
 
 const int32_t *isv_seq_lens_dev(isv_kv *h, int32_t layer) {
     if (!h || layer < 0 || layer >= h->g.layers || !h->lens_dev) return nullptr;
-    return h->lens_dev + (size_t)layer * h->g.max_seqs;
+    return lens_ptr(h, layer, 0);
 }
 
 int isv_block_table_host(isv_kv *h, int32_t *out, int32_t n_seqs, int32_t row_stride) {
@@ -801,7 +866,7 @@ int isv_set_timing(isv_kv *h, int32_t on) {
     }
     h->timing = on != 0;
     if (h->lev_created)
-        for (auto &le : h->lev) le.have_append = le.have_decode = le.have_off = false;
+        for (auto &le : h->lev) le.have_append = le.have_decode = le.have_off = le.fused_append = false;
     return ISV_OK;
 }
 
@@ -823,10 +888,8 @@ int isv_step_timing(isv_kv *h, int32_t layer, isv_step_times *out) {
     const LayerEvents *first = nullptr, *last = nullptr;
     for (int l = l0; l < l1; ++l) {
         const LayerEvents &le = h->lev[l];
-        if (le.have_append) {
-            out->append_ms += ms(le.a0, le.a1);
-            out->bytes_appended += le.bytes_app;
-        }
+        if (le.have_append) out->append_ms += ms(le.a0, le.a1);
+        if (le.have_append || le.fused_append) out->bytes_appended += le.bytes_app;
         if (!le.have_decode) continue;
         if (!first) first = &le;
         last = &le;

@@ -274,7 +274,7 @@ __device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int wf
 
 // Stage metadata words written by the producing lane before it arms the stage.
 enum { M_SEG = 0, M_SEQ, M_HG, M_NTOK, M_FLAGS, M_NC, M_WF, M_WFSLOT, M_WORDS = 8 };
-enum { F_KIND_K = 0, F_KIND_V = 1, F_KIND_END = 2, F_KIND_MASK = 3, F_LAST = 4 };
+enum { F_KIND_K = 0, F_KIND_V = 1, F_KIND_END = 2, F_KIND_NEW = 3, F_KIND_MASK = 3, F_LAST = 4 };
 
 // A split whose partial has been stored but whose arrival has not been
 // published yet (publishing needs a fence; it is cheap once the stores have
@@ -300,6 +300,41 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
 
     const int Hg = p.Hkv * p.P;
     const uint64_t block_bytes = p.block_bytes;
+    const int fused = (MODE == MODE_RESIDENT && p.k_new != nullptr) ? 1 : 0;
+
+    // ---- fused append: the rows of this step's token go to slot len % BT of block len / BT
+    // (pool, or the sequence's tail slot when that block is host-flagged).  Nothing in this launch
+    // reads those slots: the new token is attended to from k_new / v_new directly.
+    if (fused) {
+        const int rows = p.n_seqs * 2 * p.Hkv;
+        const int row_vecs = D * 2 / 16;
+        for (int r = blockIdx.x * NW + warp; r < rows; r += gridDim.x * NW) {
+            const int s = r / (2 * p.Hkv);
+            const int kv = (r / p.Hkv) & 1, h = r % p.Hkv;
+            const int len = p.lens[s];
+            const int j = len / BT, slot = len % BT;
+            const int32_t e = p.table[(size_t)s * p.table_stride + j];
+            uint8_t *base = nullptr;
+            if (e != ISV_BLOCK_NONE) {
+                if (e & ISV_BLOCK_HOST_BIT) {
+                    if (p.tail_w) base = p.tail_w + (uint64_t)s * block_bytes;
+                } else if (e >= 0 && e < p.n_pool_blocks) {
+                    base = p.pool_w + (uint64_t)e * block_bytes;
+                }
+            }
+            if (base) {
+                if (lane < row_vecs) {
+                    const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v_new : p.k_new) +
+                                         ((size_t)s * p.Hkv + h) * (D * 2) + lane * 16;
+                    uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * TILE + (size_t)slot * (D * 2) + lane * 16;
+                    *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+                }
+            } else if (lane == 0) {
+                atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+            }
+            if (kv == 0 && h == 0 && lane == 0) p.lens_out[s] = len + 1;
+        }
+    }
 
     // ---- this warp's contiguous share of the work.  Resident mode: the flat space of KV blocks
     // ordered by (sequence, head group, block), cut into equal ranges whatever the sequence lengths
@@ -308,7 +343,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     long long NU;
     if (MODE == MODE_RESIDENT) {
         for (int s = threadIdx.x; s < p.n_seqs; s += blockDim.x) {
-            const int len = p.lens[s];
+            const int len = p.lens[s] + fused;
             ubase[s + 1] = max(1, (len + BT - 1) / BT) * Hg;
         }
         if (threadIdx.x == 0) ubase[0] = 0;
@@ -354,6 +389,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     bool pu_open = false, pu_done = false;
     const uint8_t *pv_src = nullptr;    // V tile of the block whose K tile was just issued
     int pv_ntok = 0, pv_flags = 0;
+    int pn_flags = -1;                  // >= 0: a new-token stage is due after the current block
     int prod_stage = 0, inflight = 0;
     if (MODE == MODE_RESIDENT) {   // sequence of the first unit: largest s with ubase[s] <= u_next
         int lo = 0, hi = p.n_seqs - 1;
@@ -388,6 +424,11 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             pv_src = nullptr;
             return;
         }
+        if (pn_flags >= 0) {   // this step's token, read from the caller's k / v
+            emit(nullptr, 1, pn_flags);
+            pn_flags = -1;
+            return;
+        }
         while (true) {
             if (pu_mask != 0) {
                 const int i = __ffs(pu_mask) - 1;
@@ -398,9 +439,23 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
                 const uint8_t *src;
                 if (MODE == MODE_RESIDENT) {
                     const int j = pu_base + i;
-                    if (j == pu_jlast) ntok = pu_len - j * BT;
+                    if (j == pu_jlast) ntok = pu_len - j * BT - fused;   // tokens already in the cache
                     src = (e & ISV_BLOCK_HOST_BIT) ? p.tail + (uint64_t)pu_s * block_bytes
                                                    : p.pool + (uint64_t)e * block_bytes;
+                    if (fused && j == pu_jlast) {
+                        if (last) pu_open = false;
+                        if (ntok == 0) {   // the new token opens this block
+                            emit(nullptr, 1, F_KIND_NEW | (last ? F_LAST : 0));
+                            return;
+                        }
+                        pn_flags = F_KIND_NEW | (last ? F_LAST : 0);
+                        const int kvh = pu_hg / p.P;
+                        pv_src = src + (uint64_t)(p.Hkv + kvh) * TILE;
+                        pv_ntok = ntok;
+                        pv_flags = F_KIND_V;
+                        emit(src + (uint64_t)kvh * TILE, ntok, F_KIND_K);
+                        return;
+                    }
                 } else {
                     src = p.pool + (uint64_t)e * block_bytes;
                 }
@@ -451,7 +506,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             if (MODE == MODE_RESIDENT) {
                 const int x = u_next;
                 while (x >= ubase[pu_s + 1]) ++pu_s;
-                pu_len = p.lens[pu_s];
+                pu_len = p.lens[pu_s] + fused;
                 const int nblk = (pu_len + BT - 1) / BT;
                 const int nb = max(1, nblk);
                 const int r = x - ubase[pu_s];
@@ -555,6 +610,53 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             tile_scores<D, GT, BT, BF16>(tile, ntok, grp, sub, q, sc, o, m, l);
         } else if (kind == F_KIND_V) {
             tile_values<D, GT, BT, BF16>(tile, ntok, grp, sub, sc, o, m, l);
+        } else if (kind == F_KIND_NEW) {
+            // this step's token: all groups compute its scores (the shuffles need every lane), group 0 keeps it
+            const int kvh = hg / p.P;
+            const uint16_t *krow = reinterpret_cast<const uint16_t *>(p.k_new) + ((size_t)s * p.Hkv + kvh) * D;
+            const uint16_t *vrow = reinterpret_cast<const uint16_t *>(p.v_new) + ((size_t)s * p.Hkv + kvh) * D;
+            float a[GT];
+#pragma unroll
+            for (int g = 0; g < GT; ++g) a[g] = 0.f;
+#pragma unroll
+            for (int v = 0; v < D / 64; ++v) {
+                float kf[8];
+                cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(krow + v * 64 + sub * 8)), kf);
+#pragma unroll
+                for (int g = 0; g < GT; ++g)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) a[g] = fmaf(q[g][v * 8 + e], kf[e], a[g]);
+            }
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                a[g] += __shfl_xor_sync(kFull, a[g], 4);
+                a[g] += __shfl_xor_sync(kFull, a[g], 2);
+                a[g] += __shfl_xor_sync(kFull, a[g], 1);
+            }
+            if (grp == 0) {
+                float pw[GT];
+#pragma unroll
+                for (int g = 0; g < GT; ++g) {
+                    if (a[g] > m[g]) {
+                        const float r = exp2f(m[g] - a[g]);
+                        l[g] *= r;
+#pragma unroll
+                        for (int e = 0; e < E; ++e) o[g][e] *= r;
+                        m[g] = a[g];
+                    }
+                    pw[g] = exp2f(a[g] - m[g]);
+                    l[g] += pw[g];
+                }
+#pragma unroll
+                for (int v = 0; v < D / 64; ++v) {
+                    float vf[8];
+                    cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(vrow + v * 64 + sub * 8)), vf);
+#pragma unroll
+                    for (int g = 0; g < GT; ++g)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) o[g][v * 8 + e] = fmaf(pw[g], vf[e], o[g][v * 8 + e]);
+                }
+            }
         }
         __syncwarp();   // every lane is done with this stage (data and metadata) before it is refilled
         --inflight;
@@ -841,6 +943,12 @@ DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
 }  // namespace
 
 int decode_warps(int GT) { return GT == 1 ? ISV_WARPS_GT1 : 8; }
+
+int decode_default_stages(int D, int BT, int GT) {
+    const int per_stage = decode_warps(GT) * BT * D * 2;
+    const int st = (128 << 10) / per_stage;
+    return st < 2 ? 2 : (st > 12 ? 12 : st);
+}
 
 size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode) {
     const size_t tile = (size_t)BT * D * 2;

@@ -35,6 +35,12 @@ struct DecodeParams {
     const int32_t *cblk;
     int32_t cu_first;
     int32_t cu_count;
+    // fused append (resident mode, optional): when k_new is set, `lens` holds the lengths BEFORE
+    // this step's token; the kernel stores the token's K/V rows into the cache, writes lens + 1 to
+    // lens_out, and attends to the new token straight from k_new / v_new
+    const void *k_new, *v_new;  // [n_seqs][Hkv][D] 16-bit, or NULL
+    int32_t *lens_out;          // [n_seqs]
+    uint8_t *pool_w, *tail_w;   // writable aliases of pool / tail
     // inputs / outputs
     const void *q;              // [n_seqs][Hq][D] 16-bit
     void *out;                  // [n_seqs][Hq][D] 16-bit or NULL
@@ -101,6 +107,10 @@ struct MergeParams {
 
 // Warps per CTA of the decode kernel that handles GT query heads per KV tile.
 int decode_warps(int GT);
+
+// Ring depth per warp that keeps about 128 KiB of copies in flight per SM (measured on B200: deeper
+// rings lower the achieved HBM rate).
+int decode_default_stages(int D, int BT, int GT);
 
 // Bytes of dynamic shared memory the decode kernel needs for `stages` ring
 // stages (one K or V tile each) per warp.

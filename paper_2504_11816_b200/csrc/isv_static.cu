@@ -135,7 +135,7 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     const bool bf16 = dtype == ISV_BF16;
     int stages = 0;
     size_t smem = 0;
-    for (int st = 2; st <= 12; ++st) {
+    for (int st = 2; st <= decode_default_stages(head_dim, block_tokens, GT); ++st) {
         const size_t b = decode_smem_bytes(head_dim, block_tokens, GT, st, n_seqs, MODE_RESIDENT);
         if (b <= (size_t)ds.smem_optin) { stages = st; smem = b; }
     }

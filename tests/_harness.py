@@ -68,8 +68,9 @@ class Harness:
             self.shadow.fill(layer, k, v, self.lens.tolist())
 
     # ---- one decode step through separate append / attention calls
-    def step(self, f32=True, out16=True):
-        """Returns per layer (q_bits, out_f32 ndarray or None, out16 bits or None)."""
+    def step(self, f32=True, out16=True, fused=False):
+        """One decode step, layer by layer, through isv_kv_append + isv_attn_decode or (fused) through
+        isv_decode_layer.  Returns per layer (q_bits, out_f32 ndarray or None, out16 bits or None)."""
         w = self.w
         res = []
         for layer in range(w.layers):
@@ -79,8 +80,11 @@ class Harness:
             o16 = torch.zeros((w.batch, w.q_heads, w.head_dim), device="cuda",
                               dtype=W.torch_dtype(w.dtype)) if out16 else None
             torch.cuda.synchronize()
-            B.isv_kv_append(self.h, layer, kd, vd, w.batch)
-            B.isv_attn_decode(self.h, layer, qd, o16, of, None, None, w.batch)
+            if fused:
+                B.isv_decode_layer(self.h, layer, qd, kd, vd, o16, of, w.batch)
+            else:
+                B.isv_kv_append(self.h, layer, kd, vd, w.batch)
+                B.isv_attn_decode(self.h, layer, qd, o16, of, None, None, w.batch)
             B.isv_sync(self.h)
             self.shadow.append(layer, k, v)
             res.append((q, of.cpu().numpy() if f32 else None, dev_to_bits(o16) if out16 else None))
