@@ -445,6 +445,8 @@ int isv_sync(isv_kv *h, uint32_t *status_out) {
     if (status_out) *status_out = st;
     if (st != 0) {
         CU(cudaMemset(h->status_dev, 0, 4));
+        // a kernel that gave up may have left its arrival counters half way
+        CU(cudaMemset(h->tickets, 0, (size_t)h->g.max_seqs * h->g.Hkv * h->g.P * 4));
         return fail(ISV_EDEVICE_STATUS, "a kernel reported status 0x%x (%s%s)", st,
                     (st & ISV_STATUS_BAD_BLOCK_ID) ? "bad block id " : "",
                     (st & ISV_STATUS_WAIT_EXPIRED) ? "wait expired" : "");

@@ -276,6 +276,16 @@ __device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int wf
 enum { M_SEG = 0, M_SEQ, M_HG, M_NTOK, M_FLAGS, M_NC, M_WF, M_WFSLOT, M_WORDS = 8 };
 enum { F_KIND_K = 0, F_KIND_V = 1, F_KIND_END = 2, F_KIND_NEW = 3, F_KIND_MASK = 3, F_LAST = 4 };
 
+// How the flat list of `total` work items is cut into `n` equal contiguous ranges, one per warp.
+// Ranges are numbered in item order, so the ranges that meet any interval are consecutive.
+struct Partition {
+    long long total;
+    int n;
+    __device__ int first(int v) const { return (int)(total * v / n); }
+    __device__ int end(int v) const { return (int)(total * (v + 1) / n); }
+    __device__ int range_of(int x) const { return (int)((((long long)x + 1) * n - 1) / total); }   // holds item x
+};
+
 // A split whose partial has been stored but whose arrival has not been
 // published yet (publishing needs a fence; it is cheap once the stores have
 // landed, so it is done one unit later).
@@ -296,45 +306,17 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     uint8_t *after_data = smem + (size_t)NW * stages * TILE;
     uint64_t *bars = reinterpret_cast<uint64_t *>(after_data) + warp * stages;
     int32_t *meta = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * 8) + warp * stages * M_WORDS;
-    int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * (8 + 4 * M_WORDS));
+    int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * (8 + 4 * M_WORDS));   // [n_seqs + 1]
+    int32_t *slen = ubase + p.n_seqs + 1;   // [n_seqs] tokens to attend (resident mode)
+
+    // Programmatic dependent launch: let the next kernel in the stream begin its launch as this one's
+    // CTAs retire, and do not read anything an earlier kernel may have written before that kernel is done.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int Hg = p.Hkv * p.P;
     const uint64_t block_bytes = p.block_bytes;
     const int fused = (MODE == MODE_RESIDENT && p.k_new != nullptr) ? 1 : 0;
-
-    // ---- fused append: the rows of this step's token go to slot len % BT of block len / BT
-    // (pool, or the sequence's tail slot when that block is host-flagged).  Nothing in this launch
-    // reads those slots: the new token is attended to from k_new / v_new directly.
-    if (fused) {
-        const int rows = p.n_seqs * 2 * p.Hkv;
-        const int row_vecs = D * 2 / 16;
-        for (int r = blockIdx.x * NW + warp; r < rows; r += gridDim.x * NW) {
-            const int s = r / (2 * p.Hkv);
-            const int kv = (r / p.Hkv) & 1, h = r % p.Hkv;
-            const int len = p.lens[s];
-            const int j = len / BT, slot = len % BT;
-            const int32_t e = p.table[(size_t)s * p.table_stride + j];
-            uint8_t *base = nullptr;
-            if (e != ISV_BLOCK_NONE) {
-                if (e & ISV_BLOCK_HOST_BIT) {
-                    if (p.tail_w) base = p.tail_w + (uint64_t)s * block_bytes;
-                } else if (e >= 0 && e < p.n_pool_blocks) {
-                    base = p.pool_w + (uint64_t)e * block_bytes;
-                }
-            }
-            if (base) {
-                if (lane < row_vecs) {
-                    const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v_new : p.k_new) +
-                                         ((size_t)s * p.Hkv + h) * (D * 2) + lane * 16;
-                    uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * TILE + (size_t)slot * (D * 2) + lane * 16;
-                    *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
-                }
-            } else if (lane == 0) {
-                atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
-            }
-            if (kv == 0 && h == 0 && lane == 0) p.lens_out[s] = len + 1;
-        }
-    }
 
     // ---- this warp's contiguous share of the work.  Resident mode: the flat space of KV blocks
     // ordered by (sequence, head group, block), cut into equal ranges whatever the sequence lengths
@@ -344,6 +326,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     if (MODE == MODE_RESIDENT) {
         for (int s = threadIdx.x; s < p.n_seqs; s += blockDim.x) {
             const int len = p.lens[s] + fused;
+            slen[s] = len;
             ubase[s + 1] = max(1, (len + BT - 1) / BT) * Hg;
         }
         if (threadIdx.x == 0) ubase[0] = 0;
@@ -367,13 +350,15 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     } else {
         NU = (long long)p.cu_count * Hg;
     }
-    // no more ranges than items, so that every participating warp owns at least one item
-    const long long nwt = min((long long)gridDim.x * NW, NU);
     const int gw = blockIdx.x * NW + warp;
-    if (gw >= nwt) return;
-    int u_next = (int)(NU * gw / nwt);
-    const int u_end = (int)(NU * (gw + 1) / nwt);
-
+    const int nw_grid = gridDim.x * NW;
+    Partition part;
+    part.total = NU;
+    part.n = (int)min((long long)nw_grid, NU);   // no more ranges than items: every range owns at least one
+    const bool idle = gw >= part.n;   // more warps than items: this one only helps with the append
+    const int cur_range = gw;
+    int u_next = idle ? 0 : part.first(gw);
+    const int u_end = idle ? 0 : part.end(gw);
     if (lane == 0) {
         for (int st = 0; st < stages; ++st) mbar_init(smem_u32(&bars[st]), 1);
         fence_barrier_init();
@@ -381,7 +366,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     __syncwarp();
 
     // ---- producer state (identical in all lanes except `ent`)
-    int pu_seg = -1, pu_s = 0, pu_hg = 0, pu_nc = 1, pu_wf = 0, pu_wfslot = 0;
+    int pu_seg = -1, pu_s = 0, pu_hg = 0, pu_nc = 1, pu_wf = 0, pu_wfslot = 0, pu_range = 0;
+    bool pu_first = true, range_first = true;   // the open segment is / the next one will be the first of its range
     int pu_len = 0, pu_jlast = -1, pu_j0 = 0, pu_n = 0;   // entries of the open unit: [pu_j0, pu_j0 + pu_n)
     int pu_batch = 0, pu_nbatch = 0, pu_base = 0;
     uint32_t pu_mask = 0;
@@ -404,7 +390,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         if (lane == 0) {
             int32_t *mt = meta + prod_stage * M_WORDS;
             mt[M_SEG] = pu_seg; mt[M_SEQ] = pu_s; mt[M_HG] = pu_hg; mt[M_NTOK] = ntok; mt[M_FLAGS] = flags;
-            mt[M_NC] = pu_nc; mt[M_WF] = pu_wf; mt[M_WFSLOT] = pu_wfslot;
+            mt[M_NC] = pu_nc; mt[M_WF] = pu_wf;
+            mt[M_WFSLOT] = pu_wfslot | (pu_first ? 2 : 0) | (pu_range << 2);   // three fields in one word
             const uint32_t bar = smem_u32(&bars[prod_stage]);
             if (src) {
                 mbar_arrive_expect_tx(bar, TILE);
@@ -506,7 +493,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             if (MODE == MODE_RESIDENT) {
                 const int x = u_next;
                 while (x >= ubase[pu_s + 1]) ++pu_s;
-                pu_len = p.lens[pu_s] + fused;
+                pu_len = slen[pu_s];
                 const int nblk = (pu_len + BT - 1) / BT;
                 const int nb = max(1, nblk);
                 const int r = x - ubase[pu_s];
@@ -518,14 +505,16 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
                 u_next = seg_end;
                 pu_n = nblk == 0 ? 0 : n;
                 pu_jlast = nblk - 1;
+                pu_range = cur_range;
+                pu_first = range_first;
+                range_first = false;
                 if (pu_j0 == 0 && n == nb) {
-                    pu_nc = 1;                                        // this warp holds all of it
+                    pu_nc = 1;                                        // this range holds all of it
                 } else {
-                    // warps whose ranges meet [start, start + nb): warp of index i is the largest w with NU*w/nwt <= i
-                    pu_wf = (int)((((long long)start + 1) * nwt - 1) / NU);
-                    const int wl = (int)((((long long)start + nb) * nwt - 1) / NU);
-                    pu_nc = wl - pu_wf + 1;
-                    pu_wfslot = (NU * pu_wf / nwt == start) ? 0 : 1;
+                    // the ranges that meet [start, start + nb) each contribute one partial
+                    pu_wf = part.range_of(start);
+                    pu_nc = part.range_of(start + nb - 1) - pu_wf + 1;
+                    pu_wfslot = (part.first(pu_wf) == start) ? 0 : 1;
                 }
             } else {
                 const int unit = u_next++;
@@ -545,19 +534,55 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
 
     for (int i = 0; i < stages && !pu_done; ++i) produce();
 
+    // ---- fused append (placed after the first copies are in flight so that it costs no start-up time):
+    // the rows of this step's token go to slot len % BT of block len / BT
+    // (pool, or the sequence's tail slot when that block is host-flagged).  Nothing in this launch
+    // reads those slots: the new token is attended to from k_new / v_new directly.
+    if (fused) {
+        const int rows = p.n_seqs * 2 * p.Hkv;
+        const int row_vecs = D * 2 / 16;
+        for (int r = blockIdx.x * NW + warp; r < rows; r += gridDim.x * NW) {
+            const int s = r / (2 * p.Hkv);
+            const int kv = (r / p.Hkv) & 1, h = r % p.Hkv;
+            const int len = slen[s] - 1;   // length before this step's token
+            const int j = len / BT, slot = len % BT;
+            const int32_t e = p.table[(size_t)s * p.table_stride + j];
+            uint8_t *base = nullptr;
+            if (e != ISV_BLOCK_NONE) {
+                if (e & ISV_BLOCK_HOST_BIT) {
+                    if (p.tail_w) base = p.tail_w + (uint64_t)s * block_bytes;
+                } else if (e >= 0 && e < p.n_pool_blocks) {
+                    base = p.pool_w + (uint64_t)e * block_bytes;
+                }
+            }
+            if (base) {
+                if (lane < row_vecs) {
+                    const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v_new : p.k_new) +
+                                         ((size_t)s * p.Hkv + h) * (D * 2) + lane * 16;
+                    uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * TILE + (size_t)slot * (D * 2) + lane * 16;
+                    *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+                }
+            } else if (lane == 0) {
+                atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+            }
+            if (kv == 0 && h == 0 && lane == 0) p.lens_out[s] = len + 1;
+        }
+    }
+
+
     // Publishes a stored partial: fence, ticket, and the merge if this was the last split to arrive.
     PendingArrival pend{0, 0, 0, 0, 0, 0};
     auto publish = [&]() {
         if (!pend.valid) return;
         pend.valid = 0;
-        __threadfence();
-        __syncwarp();
+        __syncwarp();   // the lanes' partial stores are ordered before lane 0's release below
         int ticket = 0;
-        if (lane == 0) ticket = atomicAdd(&p.tickets[pend.ticket_idx], 1);
-        ticket = __shfl_sync(kFull, ticket, 0);
+        if (lane == 0)
+            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
+                         : "=r"(ticket) : "l"(&p.tickets[pend.ticket_idx]) : "memory");
+        ticket = __shfl_sync(kFull, ticket, 0);   // the other lanes read the partials after lane 0's acquire
         if (ticket == pend.nc - 1) {
             if (lane == 0) p.tickets[pend.ticket_idx] = 0;   // ready for the next launch
-            __threadfence();
             for (int g = 0; g < GT; ++g)
                 merge_partials_row<D, BF16>(p, pend.wf, pend.wf_slot, pend.nc, g, GT, pend.row0 + g, lane);
         }
@@ -583,7 +608,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         const int32_t *mt = meta + cons_stage * M_WORDS;
         const int seg = mt[M_SEG], s = mt[M_SEQ], hg = mt[M_HG], nc = mt[M_NC];
         const int ntok = mt[M_NTOK], flags = mt[M_FLAGS];
-        const int mt_wf = mt[M_WF], mt_wfslot = mt[M_WFSLOT];
+        const int mt_wf = mt[M_WF], mt_pack = mt[M_WFSLOT];
         const int kind = flags & F_KIND_MASK;
         if (seg != cur_seg) {
             cur_seg = seg;
@@ -736,7 +761,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             continue;
         }
         publish();   // the previous partial's arrival; its stores have long landed
-        const int slot = 2 * gw + (seg == 0 ? 0 : 1);   // an incomplete segment is the warp's first or its last
+        // an incomplete segment is the first or the last of its range: two partial slots per range
+        const int slot = 2 * (mt_pack >> 2) + ((mt_pack & 2) ? 0 : 1);
         if (grp == 0) {
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
@@ -752,7 +778,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         pend.ticket_idx = s * Hg + hg;
         pend.nc = nc;
         pend.wf = mt_wf;
-        pend.wf_slot = mt_wfslot;
+        pend.wf_slot = mt_pack & 1;
         pend.row0 = (size_t)s * p.Hq + (size_t)hg * GT;
     }
     publish();
@@ -953,7 +979,7 @@ int decode_default_stages(int D, int BT, int GT) {
 size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode) {
     const size_t tile = (size_t)BT * D * 2;
     size_t b = (size_t)decode_warps(GT) * stages * (tile + 8 + 4 * M_WORDS);
-    if (mode == MODE_RESIDENT) b += (size_t)(max_seqs + 1) * 4;
+    if (mode == MODE_RESIDENT) b += (size_t)(2 * max_seqs + 1) * 4;
     return b;
 }
 
@@ -967,8 +993,17 @@ cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int BT, bool bf1
                           int stages, size_t smem, cudaStream_t st) {
     DecodeFn fn = pick(D, GT, BT, bf16, mode);
     if (!fn) return cudaErrorInvalidValue;
-    fn<<<grid, decode_warps(GT) * 32, smem, st>>>(p, stages);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(decode_warps(GT) * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;   // see the kernel's griddepcontrol pair
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, p, stages);
 }
 
 cudaError_t launch_table_update(int32_t *table, const TableUpdateBatch &b, cudaStream_t st) {
