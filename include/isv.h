@@ -201,9 +201,10 @@ int isv_decode_step(isv_kv *h, const void *q_dev, const void *k_dev, const void 
                     void *out_dev, int32_t n_seqs);
 
 /* The same step with HOST buffers of the same shapes (pinned memory gives
- * asynchronous copies): inputs are copied to library-owned device buffers,
- * the step runs, out is copied back.  Returns after the result is in
- * out_host (synchronises). */
+ * asynchronous copies): inputs are copied to library-owned device buffers a
+ * few layers at a time on a copy stream while earlier layers compute, and
+ * each group's result is copied back as soon as it is ready.  Returns after
+ * the whole result is in out_host (synchronises). */
 int isv_decode_step_host(isv_kv *h, const void *q_host, const void *k_host,
                          const void *v_host, void *out_host, int32_t n_seqs);
 

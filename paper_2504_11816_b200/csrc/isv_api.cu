@@ -77,7 +77,8 @@ struct isv_kv {
     uint8_t *step_buf = nullptr;           // device copies of one step's q, k, v, out (host-buffer entry point)
     uint64_t hbm_pool_bytes = 0, host_pool_bytes = 0, scratch_bytes = 0;
     // streams and events
-    cudaStream_t s_compute = nullptr, s_copy = nullptr, s_off = nullptr, s_d2h = nullptr;
+    cudaStream_t s_compute = nullptr, s_copy = nullptr, s_off = nullptr, s_d2h = nullptr, s_in = nullptr;
+    std::vector<cudaEvent_t> ev_step_in, ev_step_out;   // host-buffer step: per group of layers
     bool own_compute = false;
     std::vector<cudaEvent_t> ev_ready, ev_freed;
     std::vector<char> freed_recorded;
@@ -123,6 +124,7 @@ void destroy(isv_kv *h) {
         if (h->s_copy) cudaStreamSynchronize(h->s_copy);
         if (h->s_off) cudaStreamSynchronize(h->s_off);
         if (h->s_d2h) cudaStreamSynchronize(h->s_d2h);
+        if (h->s_in) cudaStreamSynchronize(h->s_in);
         cudaFree(h->pool_hbm); cudaFree(h->tail); cudaFree(h->table_dev); cudaFree(h->lens_dev);
         cudaFree(h->status_dev); cudaFree(h->part_o); cudaFree(h->part_ml); cudaFree(h->res_o);
         cudaFree(h->res_ml); cudaFree(h->run_o); cudaFree(h->run_ml); cudaFree(h->tickets);
@@ -136,6 +138,9 @@ void destroy(isv_kv *h) {
         for (auto e : h->ev_ready) cudaEventDestroy(e);
         for (auto e : h->ev_freed) cudaEventDestroy(e);
         for (auto e : h->ev_flush) cudaEventDestroy(e);
+        for (auto e : h->ev_step_in) cudaEventDestroy(e);
+        for (auto e : h->ev_step_out) cudaEventDestroy(e);
+        if (h->s_in) cudaStreamDestroy(h->s_in);
         if (h->ev_q) cudaEventDestroy(h->ev_q);
         if (h->ev_off_done) cudaEventDestroy(h->ev_off_done);
         if (h->ev_app) cudaEventDestroy(h->ev_app);
@@ -440,6 +445,7 @@ int isv_sync(isv_kv *h, uint32_t *status_out) {
     CU(cudaStreamSynchronize(h->s_copy));
     CU(cudaStreamSynchronize(h->s_off));
     CU(cudaStreamSynchronize(h->s_d2h));
+    if (h->s_in) CU(cudaStreamSynchronize(h->s_in));
     uint32_t st = 0;
     CU(cudaMemcpy(&st, h->status_dev, 4, cudaMemcpyDeviceToHost));
     if (status_out) *status_out = st;
@@ -775,13 +781,44 @@ int isv_decode_step_host(isv_kv *h, const void *q, const void *k, const void *v,
         if ((rc = dev_alloc((void **)&h->step_buf, 2 * qs_max + 2 * ks_max, &h->scratch_bytes, "step buffers"))) return rc;
     }
     uint8_t *dq = h->step_buf, *dout = dq + qs_max, *dk = dout + qs_max, *dv = dk + ks_max;
-    const size_t qs = (size_t)g.layers * n_seqs * g.Hq * g.D * 2, ks = (size_t)g.layers * n_seqs * g.Hkv * g.D * 2;
-    CU(cudaMemcpyAsync(dk, k, ks, cudaMemcpyHostToDevice, h->s_compute));
-    CU(cudaMemcpyAsync(dv, v, ks, cudaMemcpyHostToDevice, h->s_compute));
-    CU(cudaMemcpyAsync(dq, q, qs, cudaMemcpyHostToDevice, h->s_compute));
-    if ((rc = isv_decode_step(h, dq, dk, dv, dout, n_seqs))) return rc;
-    CU(cudaMemcpyAsync(out, dout, qs, cudaMemcpyDeviceToHost, h->s_compute));
+    // Inputs travel in groups of a few layers on their own stream and results go back on the
+    // write-back stream, so that only the first group's copy and the last group's read-back are
+    // not hidden behind the attention of the other layers.
+    const int group = 4;
+    const int n_groups = (g.layers + group - 1) / group;
+    if (h->ev_step_in.empty()) {
+        h->ev_step_in.resize(n_groups);
+        h->ev_step_out.resize(n_groups);
+        for (int i = 0; i < n_groups; ++i) {
+            CU(cudaEventCreateWithFlags(&h->ev_step_in[i], cudaEventDisableTiming));
+            CU(cudaEventCreateWithFlags(&h->ev_step_out[i], cudaEventDisableTiming));
+        }
+        CU(cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking));
+    }
+    const size_t ql = (size_t)n_seqs * g.Hq * g.D * 2, kl = (size_t)n_seqs * g.Hkv * g.D * 2;   // one layer
+    // the device buffers are free once the compute stream has finished the previous call's work (it has:
+    // the previous call synchronised), and caller data already on its way is ordered by the compute stream
+    CU(cudaEventRecord(h->ev_app, h->s_compute));
+    CU(cudaStreamWaitEvent(h->s_in, h->ev_app, 0));
+    for (int gi = 0; gi < n_groups; ++gi) {
+        const int l0 = gi * group, nl = std::min(group, g.layers - l0);
+        CU(cudaMemcpyAsync(dk + l0 * kl, (const uint8_t *)k + l0 * kl, nl * kl, cudaMemcpyHostToDevice, h->s_in));
+        CU(cudaMemcpyAsync(dv + l0 * kl, (const uint8_t *)v + l0 * kl, nl * kl, cudaMemcpyHostToDevice, h->s_in));
+        CU(cudaMemcpyAsync(dq + l0 * ql, (const uint8_t *)q + l0 * ql, nl * ql, cudaMemcpyHostToDevice, h->s_in));
+        CU(cudaEventRecord(h->ev_step_in[gi], h->s_in));
+    }
+    for (int gi = 0; gi < n_groups; ++gi) {
+        const int l0 = gi * group, nl = std::min(group, g.layers - l0);
+        CU(cudaStreamWaitEvent(h->s_compute, h->ev_step_in[gi], 0));
+        for (int l = l0; l < l0 + nl; ++l)
+            if ((rc = isv_decode_layer(h, l, dq + l * ql, dk + l * kl, dv + l * kl, dout + l * ql, nullptr, n_seqs)))
+                return rc;
+        CU(cudaEventRecord(h->ev_step_out[gi], h->s_compute));
+        CU(cudaStreamWaitEvent(h->s_d2h, h->ev_step_out[gi], 0));
+        CU(cudaMemcpyAsync((uint8_t *)out + l0 * ql, dout + l0 * ql, nl * ql, cudaMemcpyDeviceToHost, h->s_d2h));
+    }
     CU(cudaStreamSynchronize(h->s_compute));
+    CU(cudaStreamSynchronize(h->s_d2h));
     return ISV_OK;
 }
 
