@@ -216,6 +216,7 @@ def run_ours(args, w):
     import torch
     import torch.distributed as dist
     from paper_2504_11816_b200 import binding as B
+    from paper_2504_11816_b200 import replicas as R
     from paper_2504_11816_b200 import workloads as W
 
     rank = int(os.environ.get("RANK", "0"))
@@ -262,16 +263,11 @@ def run_ours(args, w):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        R.barrier(dist)
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return R.max_over_ranks(x, dist, device="cuda")
 
     # -------- pass 1: device-resident inputs, no per-layer events -> `value`
     fill()
@@ -295,7 +291,7 @@ def run_ours(args, w):
     launches = B.isv_kv_info(h).kernel_launches - launches0
     status = B.isv_sync(h)
     h2d_after = B.isv_link_probe(1 << 30, 10)[0] if w.offload_frac > 0 else None
-    value = world * w.batch * K / (ms * 1e-3)
+    value = R.aggregate_tokens_per_s(w.batch, K, ms, world)
 
     # -------- pass 2: same K steps with per-layer events -> kernel durations and byte counters
     B.isv_kv_reset(h)
@@ -373,7 +369,7 @@ def run_ours(args, w):
         torch.cuda.synchronize()
         t1 = time.perf_counter()
         e2e_s = max_over_ranks(t1 - t0)
-        e2e = {"value": world * w.batch * K / e2e_s, "unit": UNIT,
+        e2e = {"value": R.aggregate_tokens_per_s(w.batch, K, e2e_s * 1e3, world), "unit": UNIT,
                "h2d_bytes_per_step": int(hq[0].numel() * 2 + hk[0].numel() * 2 + hv[0].numel() * 2),
                "d2h_bytes_per_step": int(hout.numel() * 2), "ms_per_step": e2e_s / K * 1e3,
                "api": "isv_decode_step_host (pinned host q/k/v in, out back, every step)"}

@@ -67,3 +67,66 @@ def t_task(t_pre_layer: float, t_dec_layer: float, n_layers: int, L_out: int) ->
 def tps(BS: int, L_in: int, L_out: int, t_e2e: float) -> float:
     """Eq. 1: TPS = BS * (L_in + L_out) / T_E2E."""
     return BS * (L_in + L_out) / t_e2e
+
+
+# ---------------------------------------------------------------- cost side: Eqs. 2-3, Algorithm 1, Step 4
+
+import math
+
+
+def tps_effective(tps_actual: float, tps_slo: float) -> float:
+    """Section III-A: the effective rate cannot exceed the SLO, min(TPS_actual, TPS_SLO)."""
+    return min(tps_actual, tps_slo)
+
+
+def t_task_hours(BS: int, L_in: int, L_out: int, tps_eff: float) -> float:
+    """Eq. 2: T_task = BS * (L_in + L_out) / (TPS_effective * 3600), in hours."""
+    return BS * (L_in + L_out) / (tps_eff * 3600.0)
+
+
+def cost_efficiency(tps_eff: float, t_task_h: float, vm_price: float) -> float:
+    """Eq. 3: CE = TPS_effective * 3600 / (ceil(T_task) * VM price)."""
+    return tps_eff * 3600.0 / (math.ceil(t_task_h) * vm_price)
+
+
+def offload_ratio(mem_avail: float, mem_kvcache: float) -> float:
+    """Section IV-B, case 3: C_off = 1 - Mem_avail / Mem_KVcache."""
+    return 1.0 - mem_avail / mem_kvcache
+
+
+def candidates(instances, mem_model, mem_activation, mem_kvcache, mem_kv_per_layer, p_max):
+    """Algorithm 1 (price priority).  ``instances``: iterable of (name, gpu_memory, price).
+    Returns [(name, C_off, price)] sorted by ascending price.  Steps in the paper's order:
+    price filter; available memory = GPU memory - (model + activation); no offloading if the
+    total fits; unsuitable if the weights do not fit or one layer's KV exceeds the available
+    memory; otherwise offload the fraction that does not fit."""
+    out = []
+    mem_total = mem_model + mem_activation + mem_kvcache
+    mem_base = mem_model + mem_activation
+    for name, gpu_mem, price in instances:
+        if price <= p_max:
+            avail = gpu_mem - mem_base
+            if gpu_mem >= mem_total:
+                out.append((name, 0.0, price))
+            else:
+                if gpu_mem < mem_model or mem_kv_per_layer > avail:
+                    continue
+                c_off = 1.0 - avail / mem_kvcache
+                if mem_kv_per_layer <= avail:
+                    out.append((name, c_off, price))
+    out.sort(key=lambda r: r[2])
+    return out
+
+
+def select_instance(cands, tps_slo, BS, L_in, L_out):
+    """Step 4: drop candidates with TPS < TPS_SLO, rank the rest by Eq. 3, ties go to the
+    higher TPS.  ``cands``: iterable of (name, tps, price).  Returns the ranked list of
+    (name, tps, price, CE), best first (empty if none meets the SLO)."""
+    ranked = []
+    for name, tps_, price in cands:
+        if tps_ >= tps_slo:
+            eff = tps_effective(tps_, tps_slo)
+            ce = cost_efficiency(eff, t_task_hours(BS, L_in, L_out, eff), price)
+            ranked.append((name, tps_, price, ce))
+    ranked.sort(key=lambda r: (-r[3], -r[1]))
+    return ranked
