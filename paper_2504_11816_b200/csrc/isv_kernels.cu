@@ -86,6 +86,26 @@ __device__ __forceinline__ void cvt8(const uint4 &r, float (&f)[8]) {
     }
 }
 
+// Two independent fp32 FMAs in one instruction (sm_100 packed fp32): d0 += a0 * b0, d1 += a1 * b1,
+// each rounded exactly like fmaf.  Halves the issue slots of the dot products and the weighted sums.
+__device__ __forceinline__ void ffma2(float &d0, float &d1, float a0, float a1, float b0, float b1) {
+#ifndef ISV_NO_FFMA2
+    asm("{\n"
+        ".reg .b64 ra, rb, rd;\n"
+        "mov.b64 ra, {%2, %3};\n"
+        "mov.b64 rb, {%4, %5};\n"
+        "mov.b64 rd, {%0, %1};\n"
+        "fma.rn.f32x2 rd, ra, rb, rd;\n"
+        "mov.b64 {%0, %1}, rd;\n"
+        "}\n"
+        : "+f"(d0), "+f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+#else
+    d0 = fmaf(a0, b0, d0);
+    d1 = fmaf(a1, b1, d1);
+#endif
+}
+
 template <bool BF16>
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
     if (BF16) {
@@ -124,10 +144,8 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
 #pragma unroll
             for (int g = 0; g < GT; ++g)
 #pragma unroll
-                for (int e = 0; e < 8; e += 2) {
-                    a0[g] = fmaf(q[g][v * 8 + e], kf[e], a0[g]);
-                    a1[g] = fmaf(q[g][v * 8 + e + 1], kf[e + 1], a1[g]);
-                }
+                for (int e = 0; e < 8; e += 2)
+                    ffma2(a0[g], a1[g], q[g][v * 8 + e], q[g][v * 8 + e + 1], kf[e], kf[e + 1]);
         }
 #pragma unroll
         for (int g = 0; g < GT; ++g) {
@@ -177,7 +195,8 @@ __device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp
 #pragma unroll
                 for (int g = 0; g < GT; ++g)
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) o[g][v * 8 + e] = fmaf(pw[g], vf[e], o[g][v * 8 + e]);
+                    for (int e = 0; e < 8; e += 2)
+                        ffma2(o[g][v * 8 + e], o[g][v * 8 + e + 1], pw[g], pw[g], vf[e], vf[e + 1]);
             }
         }
     }
