@@ -161,6 +161,27 @@ int isv_kv_info(isv_kv *h, isv_kv_info_t *out);
 int isv_kv_fill(isv_kv *h, int32_t layer, const void *k_dev, const void *v_dev,
                 const int32_t *lens_host, int32_t n_seqs, int32_t T);
 
+/* The same load without the final wait: returns once the work is enqueued (k_dev and v_dev must stay valid
+ * until isv_sync or isv_fill_timing).  Resident blocks are written by a kernel; the complete host-resident
+ * blocks - the share C_off of the prompt's KV that the paper's prefill stage stores to CPU memory,
+ * T_trans^p = C_off * 2 * (L_in + 1) * h1 * Precision * BS / BW_gpu->cpu (Section IV-C) - are packed into
+ * the staging ring in host-block order and stored by device-to-host copies on the write-back stream, so
+ * that the store overlaps whatever the caller computes next (the paper's Eq. 5 takes the max of both). */
+int isv_kv_fill_async(isv_kv *h, int32_t layer, const void *k_dev, const void *v_dev,
+                      const int32_t *lens_host, int32_t n_seqs, int32_t T);
+
+/* Timing of the latest isv_kv_fill / isv_kv_fill_async: store_ms is the measured T_trans^p of that layer
+ * (first to last device-to-host copy), bytes_stored its numerator counted per block.  Synchronises. */
+typedef struct {
+    float    pack_ms;          /* kernels: resident blocks, tails, packing of host blocks */
+    float    store_ms;         /* device-to-host copies, first start to last end          */
+    float    total_ms;         /* start of the load to the end of its last copy           */
+    uint64_t bytes_stored;     /* KV bytes written to the host pool                       */
+    uint64_t bytes_resident;   /* KV bytes written to GPU memory                          */
+    int32_t  n_copies;
+} isv_fill_times;
+int isv_fill_timing(isv_kv *h, isv_fill_times *out);
+
 /* Appends one token to sequences 0..n_seqs-1 of one layer at that layer's
  * current lengths (the cache growth of one decode step): k, v are device
  * arrays [n_seqs][kv_heads][head_dim].  K and V are written by one kernel; the

@@ -32,7 +32,8 @@ ISV_BLOCK_NONE = -1
 ISV_BLOCK_HOST_BIT = 1 << 30
 
 EXPORTS = [
-    "isv_kv_alloc", "isv_kv_free", "isv_kv_reset", "isv_kv_info", "isv_kv_fill", "isv_kv_append",
+    "isv_kv_alloc", "isv_kv_free", "isv_kv_reset", "isv_kv_info", "isv_kv_fill", "isv_kv_fill_async",
+    "isv_fill_timing", "isv_kv_append",
     "isv_attn_decode", "isv_decode_layer", "isv_decode_step", "isv_decode_step_host", "isv_kv_gather",
     "isv_block_table_dev", "isv_seq_lens_dev", "isv_block_table_host", "isv_seq_lens_host",
     "isv_plan_bytes", "isv_set_timing", "isv_step_timing", "isv_sync", "isv_link_probe",
@@ -87,6 +88,13 @@ class StepTimes(ctypes.Structure):
         return {name: getattr(self, name) for name, _ in self._fields_}
 
 
+class FillTimes(ctypes.Structure):
+    _fields_ = [
+        ("pack_ms", ctypes.c_float), ("store_ms", ctypes.c_float), ("total_ms", ctypes.c_float),
+        ("bytes_stored", ctypes.c_uint64), ("bytes_resident", ctypes.c_uint64), ("n_copies", ctypes.c_int32),
+    ]
+
+
 _lib = None
 
 
@@ -107,6 +115,8 @@ def lib():
     L.isv_kv_reset.argtypes = [vp]
     L.isv_kv_info.argtypes = [vp, P(KvInfo)]
     L.isv_kv_fill.argtypes = [vp, i32, vp, vp, vp, i32, i32]
+    L.isv_kv_fill_async.argtypes = [vp, i32, vp, vp, vp, i32, i32]
+    L.isv_fill_timing.argtypes = [vp, P(FillTimes)]
     L.isv_kv_append.argtypes = [vp, i32, vp, vp, i32]
     L.isv_attn_decode.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32]
     L.isv_decode_layer.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32]
@@ -188,6 +198,17 @@ def isv_kv_info(h: int) -> KvInfo:
 def isv_kv_fill(h: int, layer: int, k, v, lens_host, n_seqs: int, T: int):
     lens = np.ascontiguousarray(lens_host, dtype=np.int32)
     _check(lib().isv_kv_fill(h, layer, _ptr(k), _ptr(v), lens.ctypes.data, n_seqs, T))
+
+
+def isv_kv_fill_async(h: int, layer: int, k, v, lens_host, n_seqs: int, T: int):
+    lens = np.ascontiguousarray(lens_host, dtype=np.int32)
+    _check(lib().isv_kv_fill_async(h, layer, _ptr(k), _ptr(v), lens.ctypes.data, n_seqs, T))
+
+
+def isv_fill_timing(h: int) -> FillTimes:
+    o = FillTimes()
+    _check(lib().isv_fill_timing(h, ctypes.byref(o)))
+    return o
 
 
 def isv_kv_append(h: int, layer: int, k, v, n_seqs: int):

@@ -86,6 +86,16 @@ struct isv_kv {
     std::vector<cudaEvent_t> ev_flush;     // per physical layer
     std::vector<char> flush_recorded;
     uint64_t chunk_counter = 0;
+    // prompt write-back (device -> host) through the same ring
+    std::vector<cudaEvent_t> ev_packed, ev_stored;
+    std::vector<char> stored_recorded;
+    int32_t *owner_dev = nullptr;          // [host_cap][2]: (sequence, block) of each host block id
+    int owner_uploaded = -1;               // host blocks in use when owner_dev was last uploaded
+    uint64_t store_counter = 0;
+    cudaEvent_t ev_f0 = nullptr, ev_f1 = nullptr, ev_s0 = nullptr, ev_s1 = nullptr;   // timing of the latest fill
+    bool fill_timed = false, fill_stored = false;
+    uint64_t fill_bytes_stored = 0, fill_bytes_resident = 0;
+    int fill_copies = 0;
     PlanSlot plan_slot[kPlanSlots];
     int plan_cur = -1;
     // kernel configuration
@@ -128,7 +138,10 @@ void destroy(isv_kv *h) {
         cudaFree(h->pool_hbm); cudaFree(h->tail); cudaFree(h->table_dev); cudaFree(h->lens_dev);
         cudaFree(h->status_dev); cudaFree(h->part_o); cudaFree(h->part_ml); cudaFree(h->res_o);
         cudaFree(h->res_ml); cudaFree(h->run_o); cudaFree(h->run_ml); cudaFree(h->tickets);
-        cudaFree(h->stage); cudaFree(h->step_buf);
+        cudaFree(h->stage); cudaFree(h->step_buf); cudaFree(h->owner_dev);
+        for (auto e : h->ev_packed) cudaEventDestroy(e);
+        for (auto e : h->ev_stored) cudaEventDestroy(e);
+        for (cudaEvent_t e : {h->ev_f0, h->ev_f1, h->ev_s0, h->ev_s1}) if (e) cudaEventDestroy(e);
         if (h->pool_host) cudaFreeHost(h->pool_host);
         for (auto &ps : h->plan_slot) {
             if (ps.host) cudaFreeHost(ps.host);
@@ -418,6 +431,17 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
         CUB(cudaEventCreateWithFlags(&h->ev_ready[r], cudaEventDisableTiming));
         CUB(cudaEventCreateWithFlags(&h->ev_freed[r], cudaEventDisableTiming));
     }
+    h->ev_packed.resize(g.ring);
+    h->ev_stored.resize(g.ring);
+    h->stored_recorded.assign(g.ring, 0);
+    for (int r = 0; r < g.ring; ++r) {
+        CUB(cudaEventCreateWithFlags(&h->ev_packed[r], cudaEventDisableTiming));
+        CUB(cudaEventCreateWithFlags(&h->ev_stored[r], cudaEventDisableTiming));
+    }
+    CUB(cudaEventCreate(&h->ev_f0)); CUB(cudaEventCreate(&h->ev_f1));
+    CUB(cudaEventCreate(&h->ev_s0)); CUB(cudaEventCreate(&h->ev_s1));
+    if (g.host_cap > 0 && (rc = dev_alloc((void **)&h->owner_dev, (size_t)g.host_cap * 8, nullptr, "host block owners")))
+        return bail(rc);
     h->ev_flush.resize(g.phys_layers);
     h->flush_recorded.assign(g.phys_layers, 0);
     for (int l = 0; l < g.phys_layers; ++l) CUB(cudaEventCreateWithFlags(&h->ev_flush[l], cudaEventDisableTiming));
@@ -469,6 +493,7 @@ int isv_kv_reset(isv_kv *h) {
         CU(cudaMemset(h->lens_dev, 0, 2 * (size_t)h->g.layers * h->g.max_seqs * 4));
         CU(cudaMemset(h->tickets, 0, (size_t)h->g.max_seqs * h->g.Hkv * h->g.P * 4));
         std::fill(h->flush_recorded.begin(), h->flush_recorded.end(), 0);
+        h->owner_uploaded = -1;
     }
     h->bm.reset();
     return ISV_OK;
@@ -497,8 +522,8 @@ int isv_kv_info(isv_kv *h, isv_kv_info_t *o) {
     return ISV_OK;
 }
 
-int isv_kv_fill(isv_kv *h, int32_t layer, const void *k, const void *v, const int32_t *lens_host,
-                int32_t n_seqs, int32_t T) {
+int isv_kv_fill_async(isv_kv *h, int32_t layer, const void *k, const void *v, const int32_t *lens_host,
+                      int32_t n_seqs, int32_t T) {
     int rc = check_handle(h, layer, false);
     if (rc) return rc;
     const Geometry &g = h->g;
@@ -517,20 +542,40 @@ int isv_kv_fill(isv_kv *h, int32_t layer, const void *k, const void *v, const in
     for (int s = 0; s < n_seqs; ++s) h->bm.length(layer, s) = lens_host[s];
     if (h->plan_only) return ISV_OK;
 
+    // the table and lengths are replaced wholesale: earlier kernels must be done with them
     CU(cudaStreamSynchronize(h->s_compute));
     CU(cudaMemcpy(h->table_dev, h->bm.table.data(), h->bm.table.size() * 4, cudaMemcpyHostToDevice));
     CU(cudaMemcpy(lens_ptr(h, layer, 0), &h->bm.len[(size_t)layer * g.max_seqs],
                   (size_t)g.max_seqs * 4, cudaMemcpyHostToDevice));
+    if (h->owner_dev && h->owner_uploaded != h->bm.host_used) {
+        std::vector<int32_t> own(2 * (size_t)h->bm.host_used);
+        for (int id = 0; id < h->bm.host_used; ++id) {
+            own[2 * id] = h->bm.host_owner_s[id];
+            own[2 * id + 1] = h->bm.host_owner_j[id];
+        }
+        if (!own.empty()) CU(cudaMemcpy(h->owner_dev, own.data(), own.size() * 4, cudaMemcpyHostToDevice));
+        h->owner_uploaded = h->bm.host_used;
+    }
     const int pl = layer % g.phys_layers;
     if (h->flush_recorded[pl]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_flush[pl], 0));
+    h->fill_timed = true;
+    h->fill_stored = false;
+    h->fill_bytes_stored = h->fill_bytes_resident = 0;
+    h->fill_copies = 0;
+    CU(cudaEventRecord(h->ev_f0, h->s_compute));
     int max_blocks = 0;
-    for (int s = 0; s < n_seqs; ++s) max_blocks = std::max(max_blocks, (lens_host[s] + g.BT - 1) / g.BT);
+    uint64_t tokens = 0;
+    for (int s = 0; s < n_seqs; ++s) {
+        max_blocks = std::max(max_blocks, (lens_host[s] + g.BT - 1) / g.BT);
+        tokens += lens_host[s];
+    }
+    // resident blocks and newest blocks: straight into the HBM pool / tail slots
     if (n_seqs > 0 && max_blocks > 0) {
         FillParams p{};
         p.k = k; p.v = v;
         p.pool = h->pool_hbm + slab_hbm(h, layer);
         p.tail = h->tail ? h->tail + slab_tail(h, layer) : nullptr;
-        p.host = h->pool_host_dev ? h->pool_host_dev + slab_host(h, layer) : nullptr;
+        p.host = nullptr;   // complete host-resident blocks take the packed path below
         p.table = h->table_dev;
         p.lens = lens_ptr(h, layer, 0);
         p.status = h->status_dev;
@@ -540,15 +585,92 @@ int isv_kv_fill(isv_kv *h, int32_t layer, const void *k, const void *v, const in
         CU(launch_fill(p, h->s_compute));
         ++h->launches;
     }
+    // complete host-resident blocks: packed into the ring in host-id order by a kernel, then stored with one
+    // device-to-host copy per run of consecutive ids, on the write-back stream, ring slot by ring slot
+    if (h->owner_dev) {
+        int id = 0;
+        bool first = true;
+        auto final_block = [&](int i) {
+            const int s = h->bm.host_owner_s[i], j = h->bm.host_owner_j[i];
+            return s >= 0 && s < n_seqs && j < h->bm.newest_block(layer, s);
+        };
+        while (id < h->bm.host_used) {
+            if (!final_block(id)) { ++id; continue; }
+            int n = 1;
+            while (id + n < h->bm.host_used && n < g.chunk_blocks && final_block(id + n)) ++n;
+            const int r = (int)(h->store_counter++ % (uint64_t)g.ring);
+            uint8_t *buf = h->stage + (size_t)r * g.chunk_bytes;
+            if (h->stored_recorded[r]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_stored[r], 0));   // slot free again
+            if (h->freed_recorded[r]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_freed[r], 0));
+            PackParams pp{};
+            pp.k = k; pp.v = v;
+            pp.owner = h->owner_dev;
+            pp.dst = buf;
+            pp.first_id = id; pp.n_ids = n;
+            pp.T = T; pp.Hkv = g.Hkv; pp.D = g.D; pp.BT = g.BT;
+            pp.block_bytes = g.block_bytes;
+            CU(launch_pack(pp, h->s_compute));
+            ++h->launches;
+            CU(cudaEventRecord(h->ev_packed[r], h->s_compute));
+            CU(cudaStreamWaitEvent(h->s_d2h, h->ev_packed[r], 0));
+            if (first) {
+                CU(cudaEventRecord(h->ev_s0, h->s_d2h));
+                first = false;
+            }
+            CU(cudaMemcpyAsync(h->pool_host + slab_host(h, layer) + (size_t)id * g.block_bytes, buf,
+                               (size_t)n * g.block_bytes, cudaMemcpyDeviceToHost, h->s_d2h));
+            CU(cudaEventRecord(h->ev_stored[r], h->s_d2h));
+            h->stored_recorded[r] = 1;
+            h->fill_bytes_stored += (uint64_t)n * g.block_bytes;
+            ++h->fill_copies;
+            id += n;
+        }
+        if (!first) {
+            CU(cudaEventRecord(h->ev_s1, h->s_d2h));
+            h->fill_stored = true;
+            // the layer's next staging must see the stored blocks
+            CU(cudaEventRecord(h->ev_flush[pl], h->s_d2h));
+            h->flush_recorded[pl] = 1;
+        }
+    }
+    h->fill_bytes_resident = tokens * g.kappa - h->fill_bytes_stored;
+    CU(cudaEventRecord(h->ev_f1, h->s_compute));
     // a full, host-flagged newest block goes to the host pool right away
     std::vector<int> flush;
     for (int s = 0; s < n_seqs; ++s) {
         const int n = lens_host[s];
         if (n > 0 && n % g.BT == 0 && h->bm.is_host((n - 1) / g.BT)) flush.push_back(s);
     }
-    if ((rc = flush_tails(h, layer, flush))) return rc;
+    return flush_tails(h, layer, flush);
+}
+
+int isv_kv_fill(isv_kv *h, int32_t layer, const void *k, const void *v, const int32_t *lens_host,
+                int32_t n_seqs, int32_t T) {
+    int rc = isv_kv_fill_async(h, layer, k, v, lens_host, n_seqs, T);
+    if (rc || h->plan_only) return rc;
     CU(cudaStreamSynchronize(h->s_compute));
     CU(cudaStreamSynchronize(h->s_d2h));
+    return ISV_OK;
+}
+
+int isv_fill_timing(isv_kv *h, isv_fill_times *out) {
+    if (!h || !out) return fail(ISV_EINVAL, "null argument");
+    if (h->plan_only) return fail(ISV_ENODEVICE, "plan-only handle");
+    memset(out, 0, sizeof *out);
+    if (!h->fill_timed) return ISV_OK;
+    CU(cudaStreamSynchronize(h->s_compute));
+    CU(cudaStreamSynchronize(h->s_d2h));
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, h->ev_f0, h->ev_f1) == cudaSuccess) out->pack_ms = t;
+    out->total_ms = out->pack_ms;
+    if (h->fill_stored) {
+        if (cudaEventElapsedTime(&t, h->ev_s0, h->ev_s1) == cudaSuccess) out->store_ms = t;
+        if (cudaEventElapsedTime(&t, h->ev_f0, h->ev_s1) == cudaSuccess) out->total_ms = std::max(out->total_ms, t);
+    }
+    out->bytes_stored = h->fill_bytes_stored;
+    out->bytes_resident = h->fill_bytes_resident;
+    out->n_copies = h->fill_copies;
+    cudaGetLastError();
     return ISV_OK;
 }
 
@@ -650,6 +772,10 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
             const int r = (int)(h->chunk_counter++ % (uint64_t)g.ring);
             uint8_t *buf = h->stage + (size_t)r * g.chunk_bytes;
             if (h->freed_recorded[r]) CU(cudaStreamWaitEvent(h->s_copy, h->ev_freed[r], 0));
+            if (h->stored_recorded[r]) {   // a prompt write-back may still be reading this slot
+                CU(cudaStreamWaitEvent(h->s_copy, h->ev_stored[r], 0));
+                h->stored_recorded[r] = 0;
+            }
             CU(cudaMemcpyAsync(buf, host_slab + (size_t)ch.first_id * g.block_bytes, (size_t)ch.n_ids * g.block_bytes,
                                cudaMemcpyHostToDevice, h->s_copy));
             CU(cudaEventRecord(h->ev_ready[r], h->s_copy));

@@ -901,6 +901,7 @@ __global__ void fill_kernel(const FillParams p) {
     if (j * p.BT >= len) return;
     const int ntok = min(p.BT, len - j * p.BT);
     const int32_t e = p.table[(size_t)s * p.table_stride + j];
+    if (!p.host && e != ISV_BLOCK_NONE && (e & ISV_BLOCK_HOST_BIT) && j != (len - 1) / p.BT) return;   // stored elsewhere
     uint8_t *base = block_base(e, s, j, len, p.BT, p.pool, p.tail, p.host, p.n_pool_blocks, p.n_host_blocks,
                                p.block_bytes);
     if (!base) {
@@ -915,6 +916,26 @@ __global__ void fill_kernel(const FillParams p) {
         int r = i - kv * per_kv;
         const int h = r / (ntok * row_vecs);
         r -= h * ntok * row_vecs;
+        const int t = r / row_vecs, vec = r - t * row_vecs;
+        const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
+                             (((size_t)s * p.T + (size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
+        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + vec * 16;
+        *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+    }
+}
+
+__global__ void pack_kernel(const PackParams p) {
+    const int b = blockIdx.x;
+    const int s = p.owner[2 * (p.first_id + b)], j = p.owner[2 * (p.first_id + b) + 1];
+    const int row_bytes = p.D * 2, row_vecs = row_bytes / 16;
+    const uint32_t tile_bytes = (uint32_t)p.BT * row_bytes;
+    uint8_t *base = p.dst + (uint64_t)b * p.block_bytes;
+    const int per_kv = p.Hkv * p.BT * row_vecs;
+    for (int i = threadIdx.x; i < 2 * per_kv; i += blockDim.x) {
+        const int kv = i / per_kv;
+        int r = i - kv * per_kv;
+        const int h = r / (p.BT * row_vecs);
+        r -= h * p.BT * row_vecs;
         const int t = r / row_vecs, vec = r - t * row_vecs;
         const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
                              (((size_t)s * p.T + (size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
@@ -1045,6 +1066,12 @@ cudaError_t launch_gather(const GatherParams &p, cudaStream_t st) {
     const int nblk = (p.len + p.BT - 1) / p.BT;
     if (nblk == 0) return cudaSuccess;
     gather_kernel<<<nblk, 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pack(const PackParams &p, cudaStream_t st) {
+    if (p.n_ids <= 0) return cudaSuccess;
+    pack_kernel<<<p.n_ids, 256, 0, st>>>(p);
     return cudaGetLastError();
 }
 

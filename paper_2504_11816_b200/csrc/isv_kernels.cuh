@@ -78,12 +78,24 @@ struct AppendParams {
 
 struct FillParams {
     const void *k, *v;          // [n_seqs][T][Hkv][D]
-    uint8_t *pool, *tail, *host; // layer slabs: HBM pool, tail slots, host pool (mapped)
+    uint8_t *pool, *tail, *host; // layer slabs: HBM pool, tail slots, host pool (mapped; NULL = complete
+                                 // host blocks are stored by the caller through PackParams instead)
     const int32_t *table;
     const int32_t *lens;        // [n_seqs] device
     uint32_t *status;
     int32_t table_stride, n_pool_blocks, n_host_blocks;
     int32_t n_seqs, T, Hkv, D, BT, max_blocks;
+    uint64_t block_bytes;
+};
+
+// Packs complete host-resident blocks of a prompt into a staging buffer in host-id order, so that
+// one device-to-host copy stores the whole run.
+struct PackParams {
+    const void *k, *v;          // [n_seqs][T][Hkv][D]
+    const int32_t *owner;       // [host blocks][2]: (sequence, logical block) of each host block id
+    uint8_t *dst;               // staging buffer; block b of the run goes to dst + b * block_bytes
+    int32_t first_id, n_ids;    // the run of host block ids
+    int32_t T, Hkv, D, BT;
     uint64_t block_bytes;
 };
 
@@ -124,6 +136,7 @@ cudaError_t launch_table_update(int32_t *table, const TableUpdateBatch &b, cudaS
 cudaError_t launch_append(const AppendParams &p, cudaStream_t st);
 cudaError_t launch_fill(const FillParams &p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams &p, cudaStream_t st);
+cudaError_t launch_pack(const PackParams &p, cudaStream_t st);
 cudaError_t launch_merge(const MergeParams &p, cudaStream_t st);
 
 }  // namespace isv

@@ -258,6 +258,37 @@ def test_decode_step_entry_points_match_per_layer_calls(f):
             assert one.bytes_resident == res_b and one.total_ms <= st.total_ms + 1e-3
 
 
+@pytest.mark.parametrize("f", [0.0, 0.5, 1.0])
+def test_async_prompt_load_stores_the_offloaded_share_and_reports_it(f):
+    """isv_kv_fill_async for all layers back to back (the stores of one layer overlap the packing of the
+    next), then the byte counters of the timing query against the cache model and a bit-exact read-back."""
+    lens = [1, 16, 33, 400, 129, 64]
+    w = small(batch=len(lens), steps=2, f=f, perm=4, ctx=(1, 400), layers=3, q_heads=4, kv_heads=4, head_dim=128)
+    block = 16 * w.kv_bytes_per_token
+    with Harness(w, lens=lens, chunk_bytes=4 * block) as hz:       # small chunks: many copies, ring reuse
+        T = max(lens)
+        keep = []
+        for layer in range(w.layers):
+            k, v = W.host_prompt(w, hz.rng, T)
+            kd, vd = bits_to_dev(k, w.dtype), bits_to_dev(v, w.dtype)
+            keep.append((kd, vd))                                   # inputs stay alive until the sync
+            torch.cuda.synchronize()
+            B.isv_kv_fill_async(hz.h, layer, kd, vd, hz.lens, w.batch, T)
+            hz.shadow.fill(layer, k, v, lens)
+        ft = B.isv_fill_timing(hz.h)                                # of the last layer; synchronises
+        res_b, off_b = km.layer_step_bytes(lens, f, 16, w.kv_bytes_per_token)
+        assert ft.bytes_stored == off_b and ft.bytes_resident == res_b
+        assert (ft.n_copies > 0) == (off_b > 0) and (ft.store_ms > 0) == (off_b > 0)
+        assert ft.pack_ms > 0 and ft.total_ms >= ft.pack_ms
+        if off_b:
+            assert ft.n_copies >= off_b // (4 * block)
+        B.isv_sync(hz.h)
+        hz.check_gather()
+        for t in range(w.steps):
+            hz.check_step(hz.step(fused=True))
+        hz.check_gather()
+
+
 def test_link_probe_reports_plausible_rates():
     h2d, d2h = B.isv_link_probe(256 << 20, 3)
     assert 1.0 < h2d < 500.0 and 1.0 < d2h < 500.0
