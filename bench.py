@@ -178,7 +178,8 @@ def workload_config(w, args, info):
                      + (f"..{w.ctx_max}" if w.ctx_max != w.ctx_min else "")
                      + f" tokens, KV block {w.block_tokens}, offload {w.offload_frac:g}",
          "offload_frac": w.offload_frac, "batch": w.batch, "layers": w.layers, "accumulate": "f32",
-         "l2": "KV read per layer-step exceeds L2 (inputs larger than L2)", "parallelism": "replicas"}
+         "l2": "KV read per layer-step exceeds L2 (inputs larger than L2)", "parallelism": "replicas",
+         "offloaded_path": "zero-copy reads" if getattr(args, "zero_copy", False) else "staged through the ring"}
     if info is not None:
         c.update({"phys_layers": info.phys_layers, "max_ctas": info.max_ctas,
                   "chunk_bytes": info.chunk_bytes, "ring_depth": info.ring_depth})
@@ -240,6 +241,8 @@ def run_ours(args, w):
     h = B.isv_kv_alloc(**desc)
     info = B.isv_kv_info(h)
     td = W.torch_dtype(w.dtype)
+    if args.zero_copy:
+        B.isv_set_zero_copy(h, True)
 
     store = {"bytes": 0, "ms": 0.0, "copies": 0, "layers": 0}
 
@@ -426,6 +429,7 @@ def main():
     ap.add_argument("--offload", type=float, default=None)
     ap.add_argument("--phys-layers", type=int, default=0)
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (small profiling cases)")
+    ap.add_argument("--zero-copy", action="store_true", help="read offloaded blocks in place instead of staging them")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

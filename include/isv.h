@@ -215,6 +215,13 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q_dev, void *out_dev,
 int isv_decode_layer(isv_kv *h, int32_t layer, const void *q_dev, const void *k_dev, const void *v_dev,
                      void *out_dev, float *out_f32_dev, int32_t n_seqs);
 
+/* Second design point for the offloaded part: with on = 1 the host-resident blocks are not staged
+ * through the ring by the copy engine; the attention kernel's bulk copies read them in place from the
+ * mapped pinned pool, over the host link.  No HBM staging traffic and no copy-engine work, but the link
+ * is driven by SM-issued reads.  Results are the same; isv_step_timing then reports h2d_ms = 0 and the
+ * link time inside attn_offloaded_ms.  Off by default. */
+int isv_set_zero_copy(isv_kv *h, int32_t on);
+
 /* One decode step of all layers: isv_decode_layer for l in 0..layers-1.
  * Device arrays: q, out [layers][n_seqs][q_heads][head_dim];
  * k, v [layers][n_seqs][kv_heads][head_dim]. */

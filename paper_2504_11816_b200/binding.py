@@ -36,7 +36,7 @@ EXPORTS = [
     "isv_fill_timing", "isv_kv_append",
     "isv_attn_decode", "isv_decode_layer", "isv_decode_step", "isv_decode_step_host", "isv_kv_gather",
     "isv_block_table_dev", "isv_seq_lens_dev", "isv_block_table_host", "isv_seq_lens_host",
-    "isv_plan_bytes", "isv_set_timing", "isv_step_timing", "isv_sync", "isv_link_probe",
+    "isv_plan_bytes", "isv_set_zero_copy", "isv_set_timing", "isv_step_timing", "isv_sync", "isv_link_probe",
     "isv_attn_decode_static", "isv_last_error",
 ]
 
@@ -130,6 +130,7 @@ def lib():
     L.isv_block_table_host.argtypes = [vp, vp, i32, i32]
     L.isv_seq_lens_host.argtypes = [vp, i32, vp, i32]
     L.isv_plan_bytes.argtypes = [vp, i32, i32, P(u64), P(u64), P(u64), P(i32)]
+    L.isv_set_zero_copy.argtypes = [vp, i32]
     L.isv_set_timing.argtypes = [vp, i32]
     L.isv_step_timing.argtypes = [vp, i32, P(StepTimes)]
     L.isv_sync.argtypes = [vp, P(ctypes.c_uint32)]
@@ -268,6 +269,10 @@ def isv_plan_bytes(h: int, layer: int, n_seqs: int):
     _check(lib().isv_plan_bytes(h, layer, n_seqs, ctypes.byref(r), ctypes.byref(o), ctypes.byref(s),
                                 ctypes.byref(n)))
     return r.value, o.value, s.value, n.value
+
+
+def isv_set_zero_copy(h: int, on: bool):
+    _check(lib().isv_set_zero_copy(h, 1 if on else 0))
 
 
 def isv_set_timing(h: int, on: bool):

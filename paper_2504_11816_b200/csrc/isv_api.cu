@@ -86,6 +86,7 @@ struct isv_kv {
     std::vector<cudaEvent_t> ev_flush;     // per physical layer
     std::vector<char> flush_recorded;
     uint64_t chunk_counter = 0;
+    bool zero_copy = false;                // offloaded blocks are read in place over the host link, no staging
     // prompt write-back (device -> host) through the same ring
     std::vector<cudaEvent_t> ev_packed, ev_stored;
     std::vector<char> stored_recorded;
@@ -729,7 +730,7 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
     const bool bf16 = g.dtype == ISV_BF16;
     const int Hg = g.Hkv * g.P;
     const int nw = decode_warps(g.GT);
-    const OffPlan &pl = h->bm.plan(layer, n_seqs);
+    const OffPlan &pl = h->bm.plan(layer, n_seqs, h->zero_copy ? (1 << 30) : g.chunk_blocks);
     const bool offloaded = !pl.chunks.empty();
     const int phys = layer % g.phys_layers;
 
@@ -740,7 +741,7 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
         le->have_off = offloaded;
         le->bytes_res = pl.bytes_resident;
         le->bytes_off = pl.bytes_offloaded;
-        le->bytes_staged = offloaded ? pl.bytes_staged : 0;
+        le->bytes_staged = (offloaded && !h->zero_copy) ? pl.bytes_staged : 0;
         le->n_chunks = (int)pl.chunks.size();
         CU(cudaEventRecord(le->d0, h->s_compute));
     }
@@ -762,24 +763,32 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
         CU(cudaStreamWaitEvent(h->s_off, h->ev_q, 0));
         if ((rc = upload_plan(h, pl, &ps))) return rc;
         CU(cudaMemsetAsync(h->run_ml, 0, (size_t)n_seqs * g.Hq * 2 * 4, h->s_off));
-        if (h->flush_recorded[phys]) CU(cudaStreamWaitEvent(h->s_copy, h->ev_flush[phys], 0));
+        if (h->flush_recorded[phys]) CU(cudaStreamWaitEvent(h->zero_copy ? h->s_off : h->s_copy, h->ev_flush[phys], 0));
         if (le) {
             CU(cudaEventRecord(le->c0, h->s_copy));
             CU(cudaEventRecord(le->o0, h->s_off));
         }
         const uint8_t *host_slab = h->pool_host + slab_host(h, layer);
         for (const Chunk &ch : pl.chunks) {
-            const int r = (int)(h->chunk_counter++ % (uint64_t)g.ring);
-            uint8_t *buf = h->stage + (size_t)r * g.chunk_bytes;
-            if (h->freed_recorded[r]) CU(cudaStreamWaitEvent(h->s_copy, h->ev_freed[r], 0));
-            if (h->stored_recorded[r]) {   // a prompt write-back may still be reading this slot
-                CU(cudaStreamWaitEvent(h->s_copy, h->ev_stored[r], 0));
-                h->stored_recorded[r] = 0;
+            const uint8_t *buf;
+            int r = -1;
+            if (h->zero_copy) {
+                // the kernel's bulk copies pull the blocks straight out of mapped pinned memory
+                buf = h->pool_host_dev + slab_host(h, layer) + (size_t)ch.first_id * g.block_bytes;
+            } else {
+                r = (int)(h->chunk_counter++ % (uint64_t)g.ring);
+                uint8_t *ring_buf = h->stage + (size_t)r * g.chunk_bytes;
+                if (h->freed_recorded[r]) CU(cudaStreamWaitEvent(h->s_copy, h->ev_freed[r], 0));
+                if (h->stored_recorded[r]) {   // a prompt write-back may still be reading this slot
+                    CU(cudaStreamWaitEvent(h->s_copy, h->ev_stored[r], 0));
+                    h->stored_recorded[r] = 0;
+                }
+                CU(cudaMemcpyAsync(ring_buf, host_slab + (size_t)ch.first_id * g.block_bytes, (size_t)ch.n_ids * g.block_bytes,
+                                   cudaMemcpyHostToDevice, h->s_copy));
+                CU(cudaEventRecord(h->ev_ready[r], h->s_copy));
+                CU(cudaStreamWaitEvent(h->s_off, h->ev_ready[r], 0));
+                buf = ring_buf;
             }
-            CU(cudaMemcpyAsync(buf, host_slab + (size_t)ch.first_id * g.block_bytes, (size_t)ch.n_ids * g.block_bytes,
-                               cudaMemcpyHostToDevice, h->s_copy));
-            CU(cudaEventRecord(h->ev_ready[r], h->s_copy));
-            CU(cudaStreamWaitEvent(h->s_off, h->ev_ready[r], 0));
             DecodeParams p = base;
             p.pool = buf;
             p.n_pool_blocks = ch.n_ids;
@@ -792,11 +801,15 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
             p.acc_o = h->run_o;
             p.acc_ml = h->run_ml;
             const long long nu2 = (long long)p.cu_count * Hg;
-            const int grid = (int)std::max<long long>(1, std::min<long long>(h->sm_count, (nu2 + nw - 1) / nw));
+            // reading in place needs few CTAs to saturate the link and leaves the other SMs to the resident kernel
+            const long long cap2 = h->zero_copy ? std::max(1, h->sm_count / 4) : h->sm_count;
+            const int grid = (int)std::max<long long>(1, std::min<long long>(cap2, (nu2 + nw - 1) / nw));
             CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_STAGED, grid, h->stages_stg, h->smem_stg, h->s_off));
             ++h->launches;
-            CU(cudaEventRecord(h->ev_freed[r], h->s_off));
-            h->freed_recorded[r] = 1;
+            if (r >= 0) {
+                CU(cudaEventRecord(h->ev_freed[r], h->s_off));
+                h->freed_recorded[r] = 1;
+            }
         }
         if (le) {
             CU(cudaEventRecord(le->c1, h->s_copy));
@@ -1019,6 +1032,12 @@ int isv_plan_bytes(isv_kv *h, int32_t layer, int32_t n_seqs, uint64_t *res, uint
     if (off) *off = pl.bytes_offloaded;
     if (staged) *staged = pl.bytes_staged;
     if (n_chunks) *n_chunks = (int32_t)pl.chunks.size();
+    return ISV_OK;
+}
+
+int isv_set_zero_copy(isv_kv *h, int32_t on) {
+    if (!h) return fail(ISV_EINVAL, "null handle");
+    h->zero_copy = on != 0;
     return ISV_OK;
 }
 

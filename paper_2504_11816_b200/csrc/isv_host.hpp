@@ -66,6 +66,7 @@ struct Chunk {
 struct OffPlan {
     bool valid = false;
     int n_seqs = 0;
+    int chunk_blocks = 0;           // host blocks per chunk this plan was cut with
     std::vector<int32_t> key;       // per sequence: index of its newest block (-1 if empty)
     std::vector<Chunk> chunks;
     std::vector<int32_t> cu_seq;    // unit -> sequence
@@ -164,10 +165,11 @@ public:
     // every host block that is complete and older than its sequence's newest
     // block, grouped by staging chunk and, inside a chunk, by sequence.
     // Cached while the newest-block indices stay the same.
-    const OffPlan &plan(int layer, int n_seqs) {
+    const OffPlan &plan(int layer, int n_seqs, int chunk_blocks = 0) {
+        if (chunk_blocks <= 0) chunk_blocks = g.chunk_blocks;
         std::vector<int32_t> key(n_seqs);
         for (int s = 0; s < n_seqs; ++s) key[s] = newest_block(layer, s);
-        bool same = plan_.valid && plan_.n_seqs == n_seqs && plan_.key == key;
+        bool same = plan_.valid && plan_.n_seqs == n_seqs && plan_.chunk_blocks == chunk_blocks && plan_.key == key;
         if (same) {
             // byte counters depend on exact lengths, not only on block counts
             account(layer, n_seqs);
@@ -178,13 +180,14 @@ public:
         plan_.version = ver;
         plan_.valid = true;
         plan_.n_seqs = n_seqs;
+        plan_.chunk_blocks = chunk_blocks;
         plan_.key = key;
-        const int Bc = g.chunk_blocks;
+        const int Bc = chunk_blocks;
         std::vector<std::pair<int32_t, int32_t>> items;   // (sequence, slot) of one chunk
-        for (int c0 = 0; c0 < host_used; c0 += Bc) {
-            const int c1 = std::min(host_used, c0 + Bc);
+        for (long long c0 = 0; c0 < host_used; c0 += Bc) {
+            const int c1 = (int)std::min<long long>(host_used, c0 + Bc);
             int first = -1, last = -1;
-            for (int id = c0; id < c1; ++id) {
+            for (int id = (int)c0; id < c1; ++id) {
                 const int s = host_owner_s[id], j = host_owner_j[id];
                 if (s < 0 || s >= n_seqs || j >= key[s]) continue;
                 if (first < 0) first = id;

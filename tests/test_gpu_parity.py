@@ -57,6 +57,26 @@ def test_parity_over_offload_fractions_with_ragged_lengths(f, perm, fused):
         hz.check_gather()
 
 
+@pytest.mark.parametrize("f", [0.25, 1.0])
+def test_reading_host_blocks_in_place_gives_the_same_result(f):
+    """isv_set_zero_copy: the offloaded blocks are read over the host link by the kernel itself."""
+    lens = [0, 17, 100, 257, 640, 33]
+    w = small(batch=len(lens), steps=18, f=f, perm=6, ctx=(0, 640), layers=2, q_heads=8, kv_heads=4, head_dim=128)
+    with Harness(w, lens=lens) as hz:
+        hz.fill()
+        B.isv_set_zero_copy(hz.h, True)
+        B.isv_set_timing(hz.h, True)
+        for t in range(w.steps):
+            hz.check_step(hz.step(fused=t % 2 == 0))
+            if t == 8:
+                B.isv_set_zero_copy(hz.h, False)      # switching back and forth between steps is allowed
+            if t == 12:
+                B.isv_set_zero_copy(hz.h, True)
+        st = B.isv_step_timing(hz.h, -1)
+        assert st.bytes_staged == 0 and st.bytes_offloaded > 0 and st.attn_offloaded_ms > 0
+        hz.check_gather()
+
+
 @pytest.mark.parametrize("ctas", [1, 2, 7, 0])
 @pytest.mark.parametrize("chunk_blocks", [1, 0])
 def test_result_does_not_depend_on_split_or_chunk_size(ctas, chunk_blocks):
