@@ -279,6 +279,25 @@ int isv_sync(isv_kv *h, uint32_t *status_out);
  * that T_trans^d's BW_cpu->gpu stands for.  Allocates and frees its buffers. */
 int isv_link_probe(uint64_t bytes, int32_t reps, double *h2d_gbs, double *d2h_gbs);
 
+/* ---- decode linear layers (linear-layer term of T_compute^d) -------------- */
+
+/* y = x . w^T for a batch of M <= max_M <= 256 tokens: the QKV / output / MLP projections whose
+ * flops the paper counts as BS * (8 h1^2 + 4 h1 h2) per layer (Section IV-C, T_compute^d).  At
+ * decode batch sizes the product is bound by reading w once from HBM; it runs on the tensor cores
+ * (tcgen05, fp32 accumulation in tensor memory) so that the arithmetic keeps up with that read.
+ *   w_dev  [N][K] 16-bit row-major (the usual weight layout), N a multiple of 128, K of 64;
+ *          must stay valid and unchanged while the handle lives
+ *   x_dev  [M][K] 16-bit;  y_dev [M][N] 16-bit and / or y_f32_dev [M][N] fp32 (one may be NULL)
+ * isv_linear_create allocates split-K scratch and encodes the weight's tensor map (synchronous);
+ * isv_linear_forward enqueues one kernel on `stream` (asynchronous); isv_linear_status waits for
+ * the stream and returns ISV_EDEVICE_STATUS if a bounded wait inside the kernel expired. */
+typedef struct isv_linear isv_linear;
+int isv_linear_create(isv_linear **out, const void *w_dev, int32_t N, int32_t K, int32_t dtype,
+                      int32_t max_M, void *stream);
+int isv_linear_forward(isv_linear *l, const void *x_dev, void *y_dev, float *y_f32_dev, int32_t M);
+int isv_linear_status(isv_linear *l, uint32_t *status_out);
+int isv_linear_free(isv_linear *l);
+
 /* ---- decode attention for callers that cannot allocate ------------------- */
 
 /* Size of the fixed device array that holds this entry point's scratch.  Every

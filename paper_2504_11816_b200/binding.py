@@ -37,7 +37,8 @@ EXPORTS = [
     "isv_attn_decode", "isv_decode_layer", "isv_decode_step", "isv_decode_step_host", "isv_kv_gather",
     "isv_block_table_dev", "isv_seq_lens_dev", "isv_block_table_host", "isv_seq_lens_host",
     "isv_plan_bytes", "isv_set_zero_copy", "isv_set_timing", "isv_step_timing", "isv_sync", "isv_link_probe",
-    "isv_attn_decode_static", "isv_last_error",
+    "isv_attn_decode_static", "isv_linear_create", "isv_linear_forward", "isv_linear_status", "isv_linear_free",
+    "isv_last_error",
 ]
 
 
@@ -137,6 +138,10 @@ def lib():
     L.isv_link_probe.argtypes = [u64, i32, P(ctypes.c_double), P(ctypes.c_double)]
     L.isv_attn_decode_static.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp, vp,
                                          vp, vp]
+    L.isv_linear_create.argtypes = [P(vp), vp, i32, i32, i32, i32, vp]
+    L.isv_linear_forward.argtypes = [vp, vp, vp, vp, i32]
+    L.isv_linear_status.argtypes = [vp, P(ctypes.c_uint32)]
+    L.isv_linear_free.argtypes = [vp]
     L.isv_last_error.argtypes = []
     L.isv_last_error.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -312,6 +317,26 @@ def isv_attn_decode_static(kv_pool, n_pool_blocks: int, block_table, table_strid
                                         _ptr(seq_lens), n_seqs, max_blocks_per_seq, q_heads, kv_heads, head_dim,
                                         block_tokens, dtype, max_ctas, _ptr(q), _ptr(out), _ptr(out_f32),
                                         _ptr(status), stream or None))
+
+
+def isv_linear_create(w, N: int, K: int, dtype: int, max_M: int, stream: int = 0) -> int:
+    h = ctypes.c_void_p()
+    _check(lib().isv_linear_create(ctypes.byref(h), _ptr(w), N, K, dtype, max_M, stream or None))
+    return h.value
+
+
+def isv_linear_forward(l: int, x, y, y_f32, M: int):
+    _check(lib().isv_linear_forward(l, _ptr(x), _ptr(y), _ptr(y_f32), M))
+
+
+def isv_linear_status(l: int) -> int:
+    st = ctypes.c_uint32(0)
+    _check(lib().isv_linear_status(l, ctypes.byref(st)))
+    return st.value
+
+
+def isv_linear_free(l: int):
+    _check(lib().isv_linear_free(l))
 
 
 def desc_from_workload(w, **overrides) -> dict:

@@ -13,7 +13,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libisv.so")
-SOURCES = ["isv_kernels.cu", "isv_api.cu", "isv_static.cu"]
+SOURCES = ["isv_kernels.cu", "isv_api.cu", "isv_static.cu", "isv_linear.cu"]
 HEADERS = ["isv_kernels.cuh", "isv_host.hpp", os.path.join("..", "..", "include", "isv.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]

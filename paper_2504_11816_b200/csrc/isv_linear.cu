@@ -1,0 +1,437 @@
+// Decode linear layers (the "linear layer" term of the paper's T_compute^d, Section IV-C:
+// BS * (8 h1^2 + 4 h1 h2) flops per layer): y = x . w^T for a small batch of tokens, i.e. a
+// skinny GEMM that streams the weight matrix once.  With M <= 256 tokens it is bound by the HBM
+// read of w, but needs 2 * M flops per weight element, which only the tensor cores deliver at
+// that rate, so this is the one dense contraction of the decode step and it runs on tcgen05:
+//
+//   - the weight rows are the MMA's M dimension (128 rows per CTA), the tokens its N dimension
+//     (the batch, padded to a multiple of 16), so one instruction covers the whole batch;
+//   - operands are staged by 2-D TMA copies with the 128-byte swizzle into a shared-memory ring,
+//     issued by one thread of a producer warp; one thread of a second warp issues tcgen05.mma
+//     (kind::f16, fp32 accumulation in tensor memory) and releases ring stages with
+//     tcgen05.commit; four epilogue warps read the accumulator with tcgen05.ld;
+//   - the K dimension is split across CTAs so that every SM streams weights; the splits' fp32
+//     partials are summed in fixed order by the last CTA of a column tile to arrive.
+// Every wait is bounded; on expiry the kernel flags the status word, still frees its tensor
+// memory and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/isv.h"
+
+namespace isv {
+int set_error(int code, const char *msg);
+}
+
+namespace {
+
+constexpr int kTileN = 128;        // weight rows per CTA (MMA M)
+constexpr int kTileK = 64;         // elements per ring stage along K (one 128-byte swizzle row)
+constexpr int kMmaK = 16;          // K of one tcgen05.mma for 16-bit operands
+constexpr int kThreads = 192;      // warp 0: TMA, warp 1: MMA + tensor memory, warps 2-5: epilogue
+constexpr uint32_t kSpin = 1u << 22;
+
+int err(int code, const char *fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    return isv::set_error(code, buf);
+}
+
+// ---------------------------------------------------------------- device helpers
+
+__device__ __forceinline__ uint32_t s32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kSpin; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if (i > 256) __nanosleep(64);
+    }
+    return false;
+}
+// 2-D tiled TMA load: box of the tensor map at element coordinates (x = along K, y = row).
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand tile stored as rows of 128 bytes with the
+// 128-byte swizzle: 8-row groups are 1024 bytes apart (stride byte offset), the leading byte offset
+// is not used by swizzled K-major layouts, descriptor version 1, layout type 2 (SWIZZLE_128B).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);          // start address, bits [0,14)
+    d |= (uint64_t)1 << 16;                           // leading byte offset (ignored), bits [16,30)
+    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset, bits [32,46)
+    d |= (uint64_t)1 << 46;                           // version, bits [46,48)
+    d |= (uint64_t)2 << 61;                           // layout type, bits [61,64)
+    return d;
+}
+
+// Instruction descriptor of kind::f16: fp32 accumulator, A and B of the same 16-bit type, both K-major.
+__host__ __device__ constexpr uint32_t instr_desc(bool bf16, int mma_m, int mma_n) {
+    return (1u << 4)                                  // D format: F32
+         | ((bf16 ? 1u : 0u) << 7)                    // A format
+         | ((bf16 ? 1u : 0u) << 10)                   // B format
+         | (0u << 15) | (0u << 16)                    // A, B K-major
+         | ((uint32_t)(mma_n >> 3) << 17)             // N / 8
+         | ((uint32_t)(mma_m >> 4) << 24);            // M / 16
+}
+
+__device__ __forceinline__ void mma_f16_ss(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                           uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(tmem_d),
+        "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrives on the mbarrier once all tcgen05 operations issued so far by this thread have completed.
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+struct LinearParams {
+    void *y;                 // [M][N] 16-bit or NULL
+    float *y_f32;            // [M][N] or NULL
+    float *partials;         // [splits][M][N] fp32 (splits > 1)
+    int32_t *tickets;        // [N / 128], zero between launches
+    uint32_t *status;
+    int32_t M, N, K;
+    int32_t mma_n;           // batch padded to a multiple of 16
+    int32_t splits, kblocks_per_split;
+    int32_t stages, tmem_cols, bf16;
+};
+
+__device__ __forceinline__ void store_out(const LinearParams &p, int m, int n, float v) {
+    const size_t idx = (size_t)m * p.N + n;
+    if (p.y_f32) p.y_f32[idx] = v;
+    if (p.y) {
+        uint16_t *o = reinterpret_cast<uint16_t *>(p.y) + idx;
+        if (p.bf16) {
+            const __nv_bfloat16 h = __float2bfloat16_rn(v);
+            *o = *reinterpret_cast<const uint16_t *>(&h);
+        } else {
+            const __half h = __float2half_rn(v);
+            *o = *reinterpret_cast<const uint16_t *>(&h);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const LinearParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // the 128-byte swizzle wants tile bases on 1024-byte boundaries of the shared address space
+    uint8_t *smem = smem_raw + ((1024u - (s32(smem_raw) & 1023u)) & 1023u);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tile = blockIdx.x, split = blockIdx.y;
+    const uint32_t a_bytes = kTileN * kTileK * 2;                 // weight tile of one stage
+    const uint32_t b_bytes = (uint32_t)p.mma_n * kTileK * 2;      // activation tile of one stage
+    const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
+    uint8_t *ring = smem;                                          // 1024-byte aligned stages
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)p.stages * stage_bytes);
+    uint64_t *empty = full + p.stages;
+    uint64_t *accum_full = empty + p.stages;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(accum_full + 1);
+    volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(s32(&full[s]), 1);
+            mbar_init(s32(&empty[s]), 1);
+        }
+        mbar_init(s32(accum_full), 1);
+        *failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {   // tensor memory: power-of-two number of columns, >= 32
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(tmem_slot)), "r"(p.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int kb0 = split * p.kblocks_per_split;
+    const int kb1 = min(p.K / kTileK, kb0 + p.kblocks_per_split);
+    const int nkb = kb1 - kb0;
+
+    if (warp == 0) {
+        // ---- producer: one thread issues the TMA copies
+        if (lane == 0) {
+            for (int i = 0; i < nkb; ++i) {
+                const int s = i % p.stages;
+                if (i >= p.stages && !mbar_wait(s32(&empty[s]), ((i / p.stages) - 1) & 1)) { *failed = 1; break; }
+                if (*failed) break;
+                const uint32_t bar = s32(&full[s]);
+                uint8_t *st = ring + (size_t)s * stage_bytes;
+                mbar_expect_tx(bar, a_bytes + b_bytes);
+                tma_load_2d(s32(st), &map_w, (kb0 + i) * kTileK, n_tile * kTileN, bar);
+                tma_load_2d(s32(st + a_bytes), &map_x, (kb0 + i) * kTileK, 0, bar);
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer: one thread
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(p.bf16 != 0, kTileN, p.mma_n);
+            bool ok = true;
+            for (int i = 0; i < nkb && ok; ++i) {
+                const int s = i % p.stages;
+                ok = mbar_wait(s32(&full[s]), (i / p.stages) & 1);
+                if (!ok || *failed) { *failed = 1; ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_addr = s32(ring + (size_t)s * stage_bytes);
+                const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(a_addr + a_bytes);
+#pragma unroll
+                for (int k = 0; k < kTileK / kMmaK; ++k) {
+                    // 16 elements = 32 bytes further along K inside the swizzled row: +2 in units of 16 bytes
+                    mma_f16_ss(tmem_base, da + 2 * k, db + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                }
+                mma_commit(s32(&empty[s]));       // the stage may be refilled once these MMAs have read it
+            }
+            mma_commit(s32(accum_full));          // accumulator complete (also signals a failed run)
+        }
+    } else {
+        // ---- epilogue: warp w reads tensor-memory lanes [32 * (w % 4), +32) = weight rows of the tile
+        const int quarter = warp & 3;
+        const bool ok = mbar_wait(s32(accum_full), 0);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (!ok || *failed) {
+            if (lane == 0) atomicOr(p.status, ISV_STATUS_WAIT_EXPIRED);
+        } else {
+            const int n = n_tile * kTileN + quarter * 32 + lane;
+            for (int c0 = 0; c0 < p.mma_n; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int m = c0 + j;
+                    if (m < p.M) {
+                        const float v = __uint_as_float(r[j]);
+                        if (p.splits == 1) store_out(p, m, n, v);
+                        else p.partials[((size_t)split * p.M + m) * p.N + n] = v;
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- tear-down: everyone meets, tensor memory is returned, split partials are combined
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    }
+    if (p.splits > 1 && !*failed) {
+        __shared__ int s_last;
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int t = atomicAdd(&p.tickets[n_tile], 1);
+            s_last = (t == p.splits - 1);
+            if (s_last) p.tickets[n_tile] = 0;
+        }
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            for (int i = threadIdx.x; i < p.M * kTileN; i += kThreads) {
+                const int m = i / kTileN, n = n_tile * kTileN + (i % kTileN);
+                float acc = 0.f;
+                for (int s = 0; s < p.splits; ++s) acc += __ldcg(&p.partials[((size_t)s * p.M + m) * p.N + n]);
+                store_out(p, m, n, acc);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Map of a row-major [rows][K] 16-bit matrix with boxes of [box_rows][64] elements, 128-byte swizzle,
+// zero fill outside the matrix.
+int make_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows, bool bf16) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return err(ISV_ECUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
+                          const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return err(ISV_ECUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return ISV_OK;
+}
+
+}  // namespace
+
+struct isv_linear {
+    const void *w = nullptr;
+    int N = 0, K = 0, max_M = 0;
+    bool bf16 = false;
+    cudaStream_t stream = nullptr;
+    CUtensorMap map_w;
+    int splits = 1, kblocks_per_split = 0, mma_n_max = 16;
+    float *partials = nullptr;
+    int32_t *tickets = nullptr;
+    uint32_t *status = nullptr;
+    int smem_optin = 0;
+};
+
+extern "C" {
+
+int isv_linear_free(isv_linear *l) {
+    if (!l) return err(ISV_EINVAL, "null handle");
+    if (l->stream) cudaStreamSynchronize(l->stream);
+    cudaFree(l->partials);
+    cudaFree(l->tickets);
+    cudaFree(l->status);
+    delete l;
+    return ISV_OK;
+}
+
+int isv_linear_create(isv_linear **out, const void *w_dev, int32_t N, int32_t K, int32_t dtype, int32_t max_M,
+                      void *stream) {
+    if (!out) return err(ISV_EINVAL, "out is null");
+    *out = nullptr;
+    if (!w_dev || (reinterpret_cast<uintptr_t>(w_dev) & 15u)) return err(ISV_EINVAL, "w must be non-null, 16-byte aligned");
+    if (N < kTileN || N % kTileN != 0) return err(ISV_EINVAL, "N (%d) must be a positive multiple of %d", N, kTileN);
+    if (K < kTileK || K % kTileK != 0) return err(ISV_EINVAL, "K (%d) must be a positive multiple of %d", K, kTileK);
+    if (max_M < 1 || max_M > 256) return err(ISV_EINVAL, "max_M (%d) must be in [1, 256]", max_M);
+    if (dtype != ISV_F16 && dtype != ISV_BF16) return err(ISV_EINVAL, "dtype must be ISV_F16 or ISV_BF16");
+    isv_linear *l = new (std::nothrow) isv_linear();
+    if (!l) return err(ISV_EINVAL, "out of host memory");
+    l->w = w_dev; l->N = N; l->K = K; l->max_M = max_M; l->bf16 = dtype == ISV_BF16;
+    l->stream = static_cast<cudaStream_t>(stream);
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&l->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) { delete l; return err(ISV_ECUDA, "isv_linear_create: %s", cudaGetErrorString(e)); }
+    // split K so that about every SM streams weights, keeping at least 8 K-blocks per CTA
+    const int n_tiles = N / kTileN, kblocks = K / kTileK;
+    int splits = std::max(1, std::min((2 * sms + n_tiles - 1) / n_tiles, kblocks / 8));
+    l->kblocks_per_split = (kblocks + splits - 1) / splits;
+    l->splits = (kblocks + l->kblocks_per_split - 1) / l->kblocks_per_split;
+    l->mma_n_max = std::max(16, (max_M + 15) / 16 * 16);
+    int rc = make_map(&l->map_w, w_dev, N, K, kTileN, l->bf16);
+    if (rc) { delete l; return rc; }
+    e = cudaMalloc((void **)&l->tickets, (size_t)n_tiles * 4);
+    if (e == cudaSuccess) e = cudaMemset(l->tickets, 0, (size_t)n_tiles * 4);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&l->status, 4);
+    if (e == cudaSuccess) e = cudaMemset(l->status, 0, 4);
+    if (e == cudaSuccess && l->splits > 1) e = cudaMalloc((void **)&l->partials, (size_t)l->splits * max_M * N * 4);
+    // the kernel also has a few bytes of static shared memory: leave room for them under the limit
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, l->smem_optin - 1024);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        isv_linear_free(l);
+        return err(ISV_ENOMEM_DEVICE, "isv_linear_create: %s", cudaGetErrorString(e));
+    }
+    *out = l;
+    return ISV_OK;
+}
+
+int isv_linear_forward(isv_linear *l, const void *x_dev, void *y_dev, float *y_f32_dev, int32_t M) {
+    if (!l) return err(ISV_EINVAL, "null handle");
+    if (!x_dev || (!y_dev && !y_f32_dev)) return err(ISV_EINVAL, "x and one of y / y_f32 must be given");
+    if ((reinterpret_cast<uintptr_t>(x_dev) & 15u)) return err(ISV_EINVAL, "x must be 16-byte aligned");
+    if (M < 1 || M > l->max_M) return err(ISV_EINVAL, "M (%d) must be in [1, %d]", M, l->max_M);
+    LinearParams p{};
+    p.y = y_dev; p.y_f32 = y_f32_dev; p.partials = l->partials; p.tickets = l->tickets; p.status = l->status;
+    p.M = M; p.N = l->N; p.K = l->K;
+    p.mma_n = std::max(16, (M + 15) / 16 * 16);
+    p.splits = l->splits; p.kblocks_per_split = l->kblocks_per_split;
+    p.bf16 = l->bf16 ? 1 : 0;
+    int cols = 32;
+    while (cols < p.mma_n) cols *= 2;
+    p.tmem_cols = cols;
+    const size_t a_bytes = (size_t)kTileN * kTileK * 2, b_bytes = (size_t)p.mma_n * kTileK * 2;
+    const size_t stage_bytes = a_bytes + ((b_bytes + 1023) & ~(size_t)1023);
+    const size_t fixed = 1024 /* alignment slack */ + 1024 /* static */ + 512 /* barriers, slots */;
+    // two CTAs per SM when the stages allow it: finer waves, and both keep copies in flight
+    int stages = (int)std::min<size_t>(6, ((size_t)l->smem_optin / 2 - fixed) / stage_bytes);
+    if (stages < 3) stages = (int)std::min<size_t>(6, ((size_t)l->smem_optin - fixed) / stage_bytes);
+    if (stages < 2) return err(ISV_EINVAL, "shared memory too small for this batch");
+    p.stages = stages;
+    const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 1) * 8 + 64;
+    CUtensorMap map_x;
+    int rc = make_map(&map_x, x_dev, M, l->K, p.mma_n, l->bf16);   // rows beyond M read as zeros
+    if (rc) return rc;
+    dim3 grid(l->N / kTileN, l->splits);
+    linear_kernel<<<grid, kThreads, smem, l->stream>>>(l->map_w, map_x, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return err(ISV_ECUDA, "isv_linear_forward: %s", cudaGetErrorString(e));
+    return ISV_OK;
+}
+
+int isv_linear_status(isv_linear *l, uint32_t *status_out) {
+    if (!l || !status_out) return err(ISV_EINVAL, "null argument");
+    cudaError_t e = cudaStreamSynchronize(l->stream);
+    if (e == cudaSuccess) e = cudaMemcpy(status_out, l->status, 4, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return err(ISV_ECUDA, "isv_linear_status: %s", cudaGetErrorString(e));
+    if (*status_out) {
+        cudaMemset(l->status, 0, 4);
+        cudaMemset(l->tickets, 0, (size_t)(l->N / kTileN) * 4);
+        return err(ISV_EDEVICE_STATUS, "the linear kernel reported status 0x%x", *status_out);
+    }
+    return ISV_OK;
+}
+
+}  // extern "C"
