@@ -37,7 +37,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the resident decode kernel from one ncu capture (bytes per KV byte
 # processed), valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernels_sha1": None, "dram_bytes_per_kv_byte": None, "source": None}
+NCU_TRAFFIC = {"kernels_sha1": "84b8539e1a4e25951c6fcbcecf757ffe7556feae",
+               # (546.95 MB read + 4.86 MB written) / 539.23 MB algorithmic, 2-layer case of the same shape
+               "dram_bytes_per_kv_byte": (546.951424 + 4.858880) / 539.230208,
+               "source": "profiles/decode_kernel_c2_2layers.md"}
 
 
 def kernels_sha1() -> str:
