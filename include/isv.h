@@ -285,7 +285,7 @@ int isv_link_probe(uint64_t bytes, int32_t reps, double *h2d_gbs, double *d2h_gb
  * flops the paper counts as BS * (8 h1^2 + 4 h1 h2) per layer (Section IV-C, T_compute^d).  At
  * decode batch sizes the product is bound by reading w once from HBM; it runs on the tensor cores
  * (tcgen05, fp32 accumulation in tensor memory) so that the arithmetic keeps up with that read.
- *   w_dev  [N][K] 16-bit row-major (the usual weight layout), N a multiple of 128, K of 64;
+ *   w_dev  [N][K] 16-bit row-major (the usual weight layout), N and K multiples of 128;
  *          must stay valid and unchanged while the handle lives
  *   x_dev  [M][K] 16-bit;  y_dev [M][N] 16-bit and / or y_f32_dev [M][N] fp32 (one may be NULL)
  * isv_linear_create allocates split-K scratch and encodes the weight's tensor map (synchronous);

@@ -10,8 +10,9 @@
 //     issued by one thread of a producer warp; one thread of a second warp issues tcgen05.mma
 //     (kind::f16, fp32 accumulation in tensor memory) and releases ring stages with
 //     tcgen05.commit; four epilogue warps read the accumulator with tcgen05.ld;
-//   - the K dimension is split across CTAs so that every SM streams weights; the splits' fp32
-//     partials are summed in fixed order by the last CTA of a column tile to arrive.
+//   - the (column tile, K block) list is cut into equal ranges, one per persistent CTA, so every
+//     SM streams the same number of weight bytes; a tile shared by several CTAs is summed from
+//     their fp32 partials, in fixed order, by the last of them to arrive.
 // Every wait is bounded; on expiry the kernel flags the status word, still frees its tensor
 // memory and returns.
 #include <cuda.h>
@@ -34,7 +35,9 @@ int set_error(int code, const char *msg);
 namespace {
 
 constexpr int kTileN = 128;        // weight rows per CTA (MMA M)
-constexpr int kTileK = 64;         // elements per ring stage along K (one 128-byte swizzle row)
+constexpr int kSwzK = 64;          // elements of one 128-byte swizzle row
+constexpr int kSub = 2;            // swizzle rows (sub-tiles along K) per ring stage, fetched by one TMA copy
+constexpr int kTileK = kSwzK * kSub;   // elements per ring stage along K
 constexpr int kMmaK = 16;          // K of one tcgen05.mma for 16-bit operands
 constexpr int kThreads = 192;      // warp 0: TMA, warp 1: MMA + tensor memory, warps 2-5: epilogue
 constexpr uint32_t kSpin = 1u << 22;
@@ -71,11 +74,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return false;
 }
-// 2-D tiled TMA load: box of the tensor map at element coordinates (x = along K, y = row).
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+// 3-D tiled TMA load.  The matrices are described as [K / 64][rows][64 elements], so that one box of
+// {64, rows, kSub} lands as kSub consecutive [rows][64] sub-tiles, each in the 128-byte swizzle.
+// x = 0 always (a multiple of 8 elements, as the 16-byte rule for the innermost coordinate asks).
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int row, int kchunk, uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-        "l"(map), "r"(x), "r"(y), "r"(bar)
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+        "l"(map), "r"(0), "r"(row), "r"(kchunk), "r"(bar)
         : "memory");
 }
 
@@ -129,12 +134,11 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)
 struct LinearParams {
     void *y;                 // [M][N] 16-bit or NULL
     float *y_f32;            // [M][N] or NULL
-    float *partials;         // [splits][M][N] fp32 (splits > 1)
+    float *partials;         // [2 * grid][M][128] fp32: a CTA leaves at most two partial tiles
     int32_t *tickets;        // [N / 128], zero between launches
     uint32_t *status;
     int32_t M, N, K;
     int32_t mma_n;           // batch padded to a multiple of 16
-    int32_t splits, kblocks_per_split;
     int32_t stages, tmem_cols, bf16;
 };
 
@@ -153,34 +157,66 @@ __device__ __forceinline__ void store_out(const LinearParams &p, int m, int n, f
     }
 }
 
-__global__ void __launch_bounds__(kThreads)
+// The work is the flat list of (column tile, K block) pairs, tile-major; it is cut into equal
+// contiguous ranges, one per CTA (persistent, one CTA per SM), so every SM streams the same number
+// of weight bytes whatever the matrix shape.  A run of K blocks of one tile inside a range is a
+// segment: a segment that covers its whole tile is stored directly, otherwise its fp32 partial goes
+// to one of the CTA's two slots and the last CTA of that tile to arrive adds the partials in fixed
+// order.  The ring of TMA stages runs across segments without draining, and two accumulators in
+// tensor memory let the epilogue of one segment overlap the MMAs of the next.
+struct Cut {
+    long long total;
+    int n;
+    __device__ long long first(int c) const { return total * c / n; }
+    __device__ int range_of(long long x) const { return (int)(((x + 1) * n - 1) / total); }
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
 linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const LinearParams p) {
     extern __shared__ uint8_t smem_raw[];
     // the 128-byte swizzle wants tile bases on 1024-byte boundaries of the shared address space
     uint8_t *smem = smem_raw + ((1024u - (s32(smem_raw) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tile = blockIdx.x, split = blockIdx.y;
+    const int kblocks = p.K / kTileK;
+    Cut cut;
+    cut.total = (long long)(p.N / kTileN) * kblocks;
+    cut.n = (int)min((long long)gridDim.x, cut.total);
+    const int cta = blockIdx.x;
+    if (cta >= cut.n) return;
+    const long long f0 = cut.first(cta), f1 = cut.first(cta + 1);
+
     const uint32_t a_bytes = kTileN * kTileK * 2;                 // weight tile of one stage
     const uint32_t b_bytes = (uint32_t)p.mma_n * kTileK * 2;      // activation tile of one stage
     const uint32_t stage_bytes = a_bytes + ((b_bytes + 1023u) & ~1023u);
-    uint8_t *ring = smem;                                          // 1024-byte aligned stages
+    uint8_t *ring = smem;
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)p.stages * stage_bytes);
     uint64_t *empty = full + p.stages;
-    uint64_t *accum_full = empty + p.stages;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(accum_full + 1);
+    uint64_t *acc_full = empty + p.stages;      // [2]
+    uint64_t *acc_empty = acc_full + 2;         // [2]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
     volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    volatile int *is_last = failed + 1;
+    volatile int *ep_fail = failed + 2;   // written and read by the epilogue warps only, around their barrier
 
+    if (threadIdx.x == 32) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(s32(&full[s]), 1);
             mbar_init(s32(&empty[s]), 1);
         }
-        mbar_init(s32(accum_full), 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(s32(&acc_full[b]), 1);
+            mbar_init(s32(&acc_empty[b]), 4);   // one arrival per epilogue warp
+        }
         *failed = 0;
+        *ep_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {   // tensor memory: power-of-two number of columns, >= 32
+    if (warp == 1) {   // tensor memory: two accumulators of mma_n columns, power-of-two total
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(tmem_slot)), "r"(p.tmem_cols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -190,96 +226,141 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
 
-    const int kb0 = split * p.kblocks_per_split;
-    const int kb1 = min(p.K / kTileK, kb0 + p.kblocks_per_split);
-    const int nkb = kb1 - kb0;
-
     if (warp == 0) {
-        // ---- producer: one thread issues the TMA copies
+        // ---- producer: one thread walks the CTA's range and issues the TMA copies
         if (lane == 0) {
-            for (int i = 0; i < nkb; ++i) {
-                const int s = i % p.stages;
-                if (i >= p.stages && !mbar_wait(s32(&empty[s]), ((i / p.stages) - 1) & 1)) { *failed = 1; break; }
+            int it = 0;
+            for (long long f = f0; f < f1; ++f, ++it) {
+                const int t = (int)(f / kblocks), kb = (int)(f % kblocks);
+                const int s = it % p.stages;
+                if (it >= p.stages && !mbar_wait(s32(&empty[s]), ((it / p.stages) - 1) & 1)) { *failed = 1; break; }
                 if (*failed) break;
                 const uint32_t bar = s32(&full[s]);
                 uint8_t *st = ring + (size_t)s * stage_bytes;
                 mbar_expect_tx(bar, a_bytes + b_bytes);
-                tma_load_2d(s32(st), &map_w, (kb0 + i) * kTileK, n_tile * kTileN, bar);
-                tma_load_2d(s32(st + a_bytes), &map_x, (kb0 + i) * kTileK, 0, bar);
+                tma_load_3d(s32(st), &map_w, t * kTileN, kb * kSub, bar);
+                tma_load_3d(s32(st + a_bytes), &map_x, 0, kb * kSub, bar);
             }
         }
     } else if (warp == 1) {
-        // ---- MMA issuer: one thread
+        // ---- MMA issuer: one thread; accumulators alternate between segments
         if (lane == 0) {
             const uint32_t idesc = instr_desc(p.bf16 != 0, kTileN, p.mma_n);
+            int it = 0, g = 0;
             bool ok = true;
-            for (int i = 0; i < nkb && ok; ++i) {
-                const int s = i % p.stages;
-                ok = mbar_wait(s32(&full[s]), (i / p.stages) & 1);
-                if (!ok || *failed) { *failed = 1; ok = false; break; }
+            for (long long f = f0; f < f1 && ok; ++g) {
+                const int t = (int)(f / kblocks);
+                const long long seg_end = min(f1, (long long)(t + 1) * kblocks);
+                const int b = g & 1, u = g >> 1;
+                if (u >= 1 && !mbar_wait(s32(&acc_empty[b]), (u - 1) & 1)) { ok = false; break; }   // epilogue drained it
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_addr = s32(ring + (size_t)s * stage_bytes);
-                const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(a_addr + a_bytes);
+                const uint32_t acc = tmem_base + (uint32_t)(b * p.mma_n);
+                for (int i = 0; f < seg_end; ++f, ++it, ++i) {
+                    const int s = it % p.stages;
+                    if (!mbar_wait(s32(&full[s]), (it / p.stages) & 1) || *failed) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_addr = s32(ring + (size_t)s * stage_bytes);
 #pragma unroll
-                for (int k = 0; k < kTileK / kMmaK; ++k) {
-                    // 16 elements = 32 bytes further along K inside the swizzled row: +2 in units of 16 bytes
-                    mma_f16_ss(tmem_base, da + 2 * k, db + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    for (int sub = 0; sub < kSub; ++sub) {
+                        const uint64_t da = smem_desc_sw128(a_addr + sub * (kTileN * kSwzK * 2));
+                        const uint64_t db = smem_desc_sw128(a_addr + a_bytes + sub * (p.mma_n * kSwzK * 2));
+#pragma unroll
+                        for (int k = 0; k < kSwzK / kMmaK; ++k) {
+                            // 16 elements = 32 bytes further along K inside the swizzled row: +2 in units of 16 bytes
+                            mma_f16_ss(acc, da + 2 * k, db + 2 * k, idesc, (i > 0 || sub > 0 || k > 0) ? 1u : 0u);
+                        }
+                    }
+                    mma_commit(s32(&empty[s]));       // the stage may be refilled once these MMAs have read it
                 }
-                mma_commit(s32(&empty[s]));       // the stage may be refilled once these MMAs have read it
+                if (!ok) break;
+                mma_commit(s32(&acc_full[b]));        // this segment's accumulator is complete
             }
-            mma_commit(s32(accum_full));          // accumulator complete (also signals a failed run)
+            if (!ok) {   // a wait expired: flag it; the epilogue warps run into their own bounded waits
+                *failed = 1;
+                atomicOr(p.status, ISV_STATUS_WAIT_EXPIRED);
+            }
         }
     } else {
         // ---- epilogue: warp w reads tensor-memory lanes [32 * (w % 4), +32) = weight rows of the tile
         const int quarter = warp & 3;
-        const bool ok = mbar_wait(s32(accum_full), 0);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (!ok || *failed) {
-            if (lane == 0) atomicOr(p.status, ISV_STATUS_WAIT_EXPIRED);
-        } else {
-            const int n = n_tile * kTileN + quarter * 32 + lane;
+        const int row = quarter * 32 + lane;
+        const int et = threadIdx.x - 64;              // 0..127 among the epilogue threads
+        int g = 0;
+        for (long long f = f0; f < f1; ++g) {
+            const int t = (int)(f / kblocks);
+            const long long start = (long long)t * kblocks, seg_end = min(f1, start + kblocks);
+            const bool complete = (f == start) && (seg_end == start + kblocks);
+            const bool first_seg = (f == f0);
+            f = seg_end;
+            const int b = g & 1, u = g >> 1;
+            if (!mbar_wait(s32(&acc_full[b]), u & 1)) *ep_fail = 1;
+            asm volatile("bar.sync 1, 128;" ::: "memory");          // the four epilogue warps decide together
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (*ep_fail) {
+                if (lane == 0) atomicOr(p.status, ISV_STATUS_WAIT_EXPIRED);
+                break;
+            }
+            float *slot = p.partials + (size_t)(2 * cta + (first_seg ? 0 : 1)) * p.M * kTileN;
+            const int n = t * kTileN + row;
             for (int c0 = 0; c0 < p.mma_n; c0 += 16) {
                 uint32_t r[16];
-                tmem_ld_32x32b_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+                tmem_ld_32x32b_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.mma_n + c0), r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const int m = c0 + j;
                     if (m < p.M) {
                         const float v = __uint_as_float(r[j]);
-                        if (p.splits == 1) store_out(p, m, n, v);
-                        else p.partials[((size_t)split * p.M + m) * p.N + n] = v;
+                        if (complete) store_out(p, m, n, v);
+                        else slot[(size_t)m * kTileN + row] = v;
                     }
                 }
             }
+            // the accumulator may be overwritten by the segment after next
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(&acc_empty[b])) : "memory");
+            if (complete) continue;
+            // ---- partial tile: publish, and combine if every contributor of the tile has arrived
+            const int cf = cut.range_of(start), cl = cut.range_of(start + kblocks - 1);
+            const int nc = cl - cf + 1;
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");          // the four epilogue warps
+            if (et == 0) {
+                const int ticket = atomicAdd(&p.tickets[t], 1);
+                *is_last = (ticket == nc - 1);
+                if (*is_last) p.tickets[t] = 0;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (*is_last) {
+                __threadfence();
+                const int cf_slot = (cut.first(cf) == start) ? 0 : 1;
+                // eight tokens at a time so that their loads are in flight together
+                for (int m0 = 0; m0 < p.M; m0 += 8) {
+                    float acc[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+                    for (int c = 0; c < nc; ++c) {
+                        const int sl = c == 0 ? 2 * cf + cf_slot : 2 * (cf + c);
+                        const float *src = p.partials + ((size_t)sl * p.M + m0) * kTileN + et;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (m0 + j < p.M) acc[j] += __ldcg(src + (size_t)j * kTileN);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (m0 + j < p.M) store_out(p, m0 + j, t * kTileN + et, acc[j]);
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");          // is_last is reused by the next partial
         }
     }
 
-    // ---- tear-down: everyone meets, tensor memory is returned, split partials are combined
+    // ---- tear-down: everyone meets, tensor memory is returned
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
-    }
-    if (p.splits > 1 && !*failed) {
-        __shared__ int s_last;
-        __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            const int t = atomicAdd(&p.tickets[n_tile], 1);
-            s_last = (t == p.splits - 1);
-            if (s_last) p.tickets[n_tile] = 0;
-        }
-        __syncthreads();
-        if (s_last) {
-            __threadfence();
-            for (int i = threadIdx.x; i < p.M * kTileN; i += kThreads) {
-                const int m = i / kTileN, n = n_tile * kTileN + (i % kTileN);
-                float acc = 0.f;
-                for (int s = 0; s < p.splits; ++s) acc += __ldcg(&p.partials[((size_t)s * p.M + m) * p.N + n]);
-                store_out(p, m, n, acc);
-            }
-        }
     }
 }
 
@@ -301,16 +382,16 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// Map of a row-major [rows][K] 16-bit matrix with boxes of [box_rows][64] elements, 128-byte swizzle,
-// zero fill outside the matrix.
+// Map of a row-major [rows][K] 16-bit matrix seen as [K / 64][rows][64], boxes of kSub x box_rows x 64
+// elements, 128-byte swizzle, zero fill outside the matrix.
 int make_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows, bool bf16) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return err(ISV_ECUDA, "cuTensorMapEncodeTiled is not available from this driver");
-    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
+    const cuuint64_t dims[3] = {(cuuint64_t)kSwzK, (cuuint64_t)rows, (cuuint64_t)(K / kSwzK)};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)kSwzK * 2};   // bytes: next row, next 64-element chunk
+    const cuuint32_t box[3] = {(cuuint32_t)kSwzK, (cuuint32_t)box_rows, (cuuint32_t)kSub};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
                           const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -326,7 +407,7 @@ struct isv_linear {
     bool bf16 = false;
     cudaStream_t stream = nullptr;
     CUtensorMap map_w;
-    int splits = 1, kblocks_per_split = 0, mma_n_max = 16;
+    int grid = 1;
     float *partials = nullptr;
     int32_t *tickets = nullptr;
     uint32_t *status = nullptr;
@@ -363,19 +444,15 @@ int isv_linear_create(isv_linear **out, const void *w_dev, int32_t N, int32_t K,
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&l->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     if (e != cudaSuccess) { delete l; return err(ISV_ECUDA, "isv_linear_create: %s", cudaGetErrorString(e)); }
-    // split K so that about every SM streams weights, keeping at least 8 K-blocks per CTA
-    const int n_tiles = N / kTileN, kblocks = K / kTileK;
-    int splits = std::max(1, std::min((2 * sms + n_tiles - 1) / n_tiles, kblocks / 8));
-    l->kblocks_per_split = (kblocks + splits - 1) / splits;
-    l->splits = (kblocks + l->kblocks_per_split - 1) / l->kblocks_per_split;
-    l->mma_n_max = std::max(16, (max_M + 15) / 16 * 16);
+    const int n_tiles = N / kTileN;
+    l->grid = sms;                      // persistent: one CTA per SM
     int rc = make_map(&l->map_w, w_dev, N, K, kTileN, l->bf16);
     if (rc) { delete l; return rc; }
     e = cudaMalloc((void **)&l->tickets, (size_t)n_tiles * 4);
     if (e == cudaSuccess) e = cudaMemset(l->tickets, 0, (size_t)n_tiles * 4);
     if (e == cudaSuccess) e = cudaMalloc((void **)&l->status, 4);
     if (e == cudaSuccess) e = cudaMemset(l->status, 0, 4);
-    if (e == cudaSuccess && l->splits > 1) e = cudaMalloc((void **)&l->partials, (size_t)l->splits * max_M * N * 4);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&l->partials, (size_t)2 * l->grid * max_M * kTileN * 4);
     // the kernel also has a few bytes of static shared memory: leave room for them under the limit
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, l->smem_optin - 1024);
@@ -397,25 +474,21 @@ int isv_linear_forward(isv_linear *l, const void *x_dev, void *y_dev, float *y_f
     p.y = y_dev; p.y_f32 = y_f32_dev; p.partials = l->partials; p.tickets = l->tickets; p.status = l->status;
     p.M = M; p.N = l->N; p.K = l->K;
     p.mma_n = std::max(16, (M + 15) / 16 * 16);
-    p.splits = l->splits; p.kblocks_per_split = l->kblocks_per_split;
     p.bf16 = l->bf16 ? 1 : 0;
     int cols = 32;
-    while (cols < p.mma_n) cols *= 2;
+    while (cols < 2 * p.mma_n) cols *= 2;        // two accumulators
     p.tmem_cols = cols;
     const size_t a_bytes = (size_t)kTileN * kTileK * 2, b_bytes = (size_t)p.mma_n * kTileK * 2;
     const size_t stage_bytes = a_bytes + ((b_bytes + 1023) & ~(size_t)1023);
     const size_t fixed = 1024 /* alignment slack */ + 1024 /* static */ + 512 /* barriers, slots */;
-    // two CTAs per SM when the stages allow it: finer waves, and both keep copies in flight
-    int stages = (int)std::min<size_t>(6, ((size_t)l->smem_optin / 2 - fixed) / stage_bytes);
-    if (stages < 3) stages = (int)std::min<size_t>(6, ((size_t)l->smem_optin - fixed) / stage_bytes);
+    int stages = (int)std::min<size_t>(std::max<size_t>(3, (160u << 10) / stage_bytes), ((size_t)l->smem_optin - fixed) / stage_bytes);
     if (stages < 2) return err(ISV_EINVAL, "shared memory too small for this batch");
     p.stages = stages;
-    const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 1) * 8 + 64;
+    const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 4) * 8 + 64;
     CUtensorMap map_x;
     int rc = make_map(&map_x, x_dev, M, l->K, p.mma_n, l->bf16);   // rows beyond M read as zeros
     if (rc) return rc;
-    dim3 grid(l->N / kTileN, l->splits);
-    linear_kernel<<<grid, kThreads, smem, l->stream>>>(l->map_w, map_x, p);
+    linear_kernel<<<l->grid, kThreads, smem, l->stream>>>(l->map_w, map_x, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return err(ISV_ECUDA, "isv_linear_forward: %s", cudaGetErrorString(e));
     return ISV_OK;

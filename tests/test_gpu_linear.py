@@ -21,7 +21,7 @@ def _case(M, N, K, dtype, seed):
 
 
 @pytest.mark.parametrize("M,N,K,dtype", [
-    (1, 128, 64, "f16"), (5, 256, 512, "f16"), (16, 128, 1024, "bf16"), (32, 512, 4096, "f16"),
+    (1, 128, 128, "f16"), (5, 256, 512, "f16"), (16, 128, 1024, "bf16"), (32, 512, 4096, "f16"),
     (33, 384, 2048, "bf16"), (100, 256, 1024, "f16"), (256, 256, 512, "f16"), (64, 1408, 1024, "bf16"),
 ])
 def test_linear_matches_reference(M, N, K, dtype):
@@ -51,12 +51,12 @@ def test_linear_matches_reference(M, N, K, dtype):
 
 
 def test_linear_rejects_bad_shapes():
-    w = torch.zeros((128, 64), device="cuda", dtype=torch.float16)
-    for N, K, maxM in ((100, 64, 16), (128, 60, 16), (128, 64, 300), (0, 64, 16)):
+    w = torch.zeros((128, 128), device="cuda", dtype=torch.float16)
+    for N, K, maxM in ((100, 128, 16), (128, 64, 16), (128, 128, 300), (0, 128, 16)):
         with pytest.raises(B.IsvError) as ei:
             B.isv_linear_create(w, N, K, B.ISV_F16, maxM, 0)
         assert ei.value.code == B.ISV_EINVAL
-    l = B.isv_linear_create(w, 128, 64, B.ISV_F16, 16, 0)
+    l = B.isv_linear_create(w, 128, 128, B.ISV_F16, 16, 0)
     try:
         with pytest.raises(B.IsvError):
             B.isv_linear_forward(l, w, w, None, 17)
