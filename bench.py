@@ -443,7 +443,7 @@ def main():
     if args.layers is not None:
         w = w.with_(layers=args.layers)
     if args.steps is None:
-        args.steps = 64 if args.impl == "ours" and w.offload_frac == 0 else (5 if args.impl == "reference" else 4)
+        args.steps = 128 if args.impl == "ours" and w.offload_frac == 0 else (5 if args.impl == "reference" else 4)
     if args.warmup < 0 or args.steps < 1:
         raise SystemExit("steps must be >= 1 and warmup >= 0")
     if args.impl == "reference":

@@ -5,7 +5,8 @@
 Follows the paper's procedure (Section IV-E): run the workload at several
 batch sizes, take the measured per-layer time from ``isv_step_timing``, and
 fit CTCF(T) = alpha * T + beta by least squares against the model's
-T_compute^d attention term (4 * BS * ctx * h1 / FLOPS).  A second run with part
+T_compute^d attention term (4 * BS * ctx * h1 / FLOPS), and against the whole
+T_compute^d with the linear layers measured through isv_linear_forward.  A second run with part
 of the cache offloaded compares the measured host-link time with the model's
 T_trans^d for the measured link bandwidth, and the measured step time with
 Eq. 6 (sum) and with the overlapped alternative (max).  Prints one JSON
@@ -59,6 +60,41 @@ def measure(w, steps: int, warmup: int):
         B.isv_kv_free(h)
 
 
+def measure_linear(h1: int, h2: int, batch: int, iters: int = 20) -> float:
+    """Seconds per layer of the four decode projections (fused QKV, output, MLP up, MLP down) through
+    isv_linear_forward, weights cycled through more than L2."""
+    import torch
+    from . import binding as B
+    stream = torch.cuda.Stream()
+    total = 0.0
+    for N, K in ((3 * h1, h1), (h1, h1), (h2, h1), (h1, h2)):
+        copies = max(2, int((384 << 20) // (N * K * 2)) + 1)
+        g = torch.Generator(device="cuda")
+        g.manual_seed(N * 131 + K)
+        ws = [(torch.randn((N, K), generator=g, device="cuda") / K ** 0.5).half() for _ in range(copies)]
+        x = torch.randn((batch, K), generator=g, device="cuda").half()
+        y = torch.zeros((batch, N), device="cuda", dtype=torch.float16)
+        torch.cuda.synchronize()
+        hs = [B.isv_linear_create(w, N, K, B.ISV_F16, max(batch, 16), stream.cuda_stream) for w in ws]
+        try:
+            for h in hs:
+                B.isv_linear_forward(h, x, y, None, batch)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(iters):
+                B.isv_linear_forward(hs[i % copies], x, y, None, batch)
+            e1.record(stream)
+            stream.synchronize()
+            assert B.isv_linear_status(hs[0]) == 0
+            total += e0.elapsed_time(e1) * 1e-3 / iters
+        finally:
+            for h in hs:
+                B.isv_linear_free(h)
+        del ws
+        torch.cuda.empty_cache()
+    return total
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--ctx", type=int, default=512)
@@ -83,14 +119,22 @@ def main():
         m = measure(base.with_(batch=bs), steps, warmup)
         ctx_mean = args.ctx + warmup + (steps + 1) / 2.0
         model_attn = 4.0 * bs * ctx_mean * shape.h1 / hw.flops          # attention term of T_compute^d
+        lin_meas = measure_linear(shape.h1, shape.h2, bs)
+        lin_model = bs * (8.0 * shape.h1 ** 2 + 4.0 * shape.h1 * shape.h2) / hw.flops      # linear term of T_compute^d
         rows.append({"batch": bs, "model_attn_s": model_attn, "measured_attn_s": m["attn"],
-                     "hbm_GBps": m["bytes_res"] / m["attn"] / 1e9})
+                     "hbm_GBps": m["bytes_res"] / m["attn"] / 1e9,
+                     "model_linear_s": lin_model, "measured_linear_s": lin_meas})
         t_model.append(model_attn)
         t_meas.append(m["attn"])
     alpha, beta, err = cm.fit_ctcf(t_model, t_meas)
+    # the paper calibrates the whole T_compute^d (linear + attention) with one line
+    alpha_c, beta_c, err_c = cm.fit_ctcf([r["model_attn_s"] + r["model_linear_s"] for r in rows],
+                                         [r["measured_attn_s"] + r["measured_linear_s"] for r in rows])
     for r in rows:
         r["ctcf_s"] = cm.ctcf(r["model_attn_s"], alpha, beta)
         r["error_pct"] = abs(r["ctcf_s"] - r["measured_attn_s"]) / r["measured_attn_s"] * 100
+        r["t_compute_d_measured_s"] = r["measured_attn_s"] + r["measured_linear_s"]
+        r["t_compute_d_ctcf_s"] = cm.ctcf(r["model_attn_s"] + r["model_linear_s"], alpha_c, beta_c)
     # offloaded run: transfer term and the sum-vs-max question
     bs = 32
     off = measure(base.with_(batch=bs, offload_frac=args.offload), 4, 3)
@@ -99,7 +143,10 @@ def main():
     result = {
         "device": torch.cuda.get_device_name(0), "link_GBps": {"h2d": h2d, "d2h": d2h},
         "shape": {"h1": shape.h1, "layers": base.layers, "ctx": args.ctx, "out_len": args.out_len},
-        "flops_used": hw.flops, "ctcf": {"alpha": alpha, "beta_s": beta, "avg_error_pct": err}, "rows": rows,
+        "flops_used": hw.flops, "ctcf": {"alpha": alpha, "beta_s": beta, "avg_error_pct": err},
+        "ctcf_full_compute": {"alpha": alpha_c, "beta_s": beta_c, "avg_error_pct": err_c,
+                              "what": "T_compute^d = linear + attention, both measured on this library"},
+        "rows": rows,
         "offloaded": {"batch": bs, "offload_frac": args.offload, "bytes_off_per_layer": off["bytes_off"],
                       "t_trans_model_s": model_trans, "t_trans_measured_s": off["h2d"],
                       "t_layer_measured_s": off["total"],
