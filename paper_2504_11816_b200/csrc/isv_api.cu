@@ -719,7 +719,7 @@ int isv_kv_append(isv_kv *h, int32_t layer, const void *k, const void *v, int32_
 // (the device lengths then still hold the values before the append and the kernel advances them).
 static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float *out_f32,
                        const int32_t *block_table_dev, const int32_t *seq_lens_dev, int32_t n_seqs,
-                       const void *k_new, const void *v_new) {
+                       const void *k_new, const void *v_new, bool tables_settled) {
     int rc = ISV_OK;
     const Geometry &g = h->g;
     if (n_seqs < 0 || n_seqs > g.max_seqs) return fail(ISV_EINVAL, "n_seqs %d outside [0, %d]", n_seqs, g.max_seqs);
@@ -835,6 +835,9 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
             p.lens_out = lens_ptr(h, layer, 1);
             p.pool_w = h->pool_hbm + slab_hbm(h, layer);
             p.tail_w = h->tail ? h->tail + slab_tail(h, layer) : nullptr;
+            // the kernel launched just before this one (the previous layer's, or a caller's) writes neither
+            // the table, nor these lengths, nor this layer's slab: their reads need not wait for it
+            p.early_reads = (tables_settled && g.phys_layers > 1) ? 1 : 0;
         }
         long long nu = 0;   // KV blocks in the flat work list
         for (int s = 0; s < n_seqs; ++s)
@@ -867,7 +870,7 @@ int isv_attn_decode(isv_kv *h, int32_t layer, const void *q, void *out, float *o
                     const int32_t *block_table_dev, const int32_t *seq_lens_dev, int32_t n_seqs) {
     int rc = check_handle(h, layer, true);
     if (rc) return rc;
-    return decode_impl(h, layer, q, out, out_f32, block_table_dev, seq_lens_dev, n_seqs, nullptr, nullptr);
+    return decode_impl(h, layer, q, out, out_f32, block_table_dev, seq_lens_dev, n_seqs, nullptr, nullptr, false);
 }
 
 int isv_decode_layer(isv_kv *h, int32_t layer, const void *q, const void *k, const void *v, void *out,
@@ -888,7 +891,7 @@ int isv_decode_layer(isv_kv *h, int32_t layer, const void *q, const void *k, con
     if ((rc = push_updates(h, ap.upd))) return rc;
     const int pl = layer % g.phys_layers;
     if (ap.new_host_block && h->flush_recorded[pl]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_flush[pl], 0));
-    if ((rc = decode_impl(h, layer, q, out, out_f32, nullptr, nullptr, n_seqs, k, v))) return rc;
+    if ((rc = decode_impl(h, layer, q, out, out_f32, nullptr, nullptr, n_seqs, k, v, ap.upd.empty()))) return rc;
     if (h->timing) h->lev[layer].bytes_app = (uint64_t)n_seqs * g.kappa;
     return flush_tails(h, layer, ap.flush);
 }

@@ -330,8 +330,13 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
 
     // Programmatic dependent launch: let the next kernel in the stream begin its launch as this one's
     // CTAs retire, and do not read anything an earlier kernel may have written before that kernel is done.
+    // With early_reads the wait is postponed until after the first K/V copies are issued: lengths, block
+    // table and this layer's KV slab were last written by kernels that finished long ago (only the kernel
+    // launched immediately before may still be running, and the host sets the flag only when that kernel
+    // writes none of them), whereas q, the new K/V rows, the scratch and the outputs are touched only
+    // after the wait.  The pipeline's ramp-up then overlaps the previous kernel's tail.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!p.early_reads) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int Hg = p.Hkv * p.P;
     const uint64_t block_bytes = p.block_bytes;
@@ -552,6 +557,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     };
 
     for (int i = 0; i < stages && !pu_done; ++i) produce();
+    if (p.early_reads) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- fused append (placed after the first copies are in flight so that it costs no start-up time):
     // the rows of this step's token go to slot len % BT of block len / BT

@@ -54,6 +54,7 @@ struct DecodeParams {
     uint32_t *status;
     int32_t n_seqs, Hq, Hkv, P;
     int32_t finalize;           // resident: 1 = normalise and write out; 0 = leave (m, l, o) in acc_*
+    int32_t early_reads;        // 1 = lengths, table and KV may be read before the dependency wait
     float scale_log2;           // log2(e) / sqrt(D)
     uint64_t block_bytes;
 };
