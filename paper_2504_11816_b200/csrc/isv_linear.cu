@@ -171,7 +171,7 @@ struct Cut {
     __device__ int range_of(long long x) const { return (int)(((x + 1) * n - 1) / total); }
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const LinearParams p) {
     extern __shared__ uint8_t smem_raw[];
     // the 128-byte swizzle wants tile bases on 1024-byte boundaries of the shared address space
@@ -225,15 +225,31 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ---- producer: one thread walks the CTA's range and issues the TMA copies
         if (lane == 0) {
-            int it = 0;
-            for (long long f = f0; f < f1; ++f, ++it) {
+            // The weights never change, so the ring is first filled with weight tiles; only then does the
+            // producer wait for the kernels launched before this one (programmatic dependent launch) and
+            // fetch the matching activation tiles.  The ramp-up thus overlaps the previous kernel's tail.
+            const int prefill = (int)min((long long)p.stages, f1 - f0);
+            for (int it = 0; it < prefill; ++it) {
+                const long long f = f0 + it;
+                const uint32_t bar = s32(&full[it]);
+                mbar_expect_tx(bar, a_bytes + b_bytes);
+                tma_load_3d(s32(ring + (size_t)it * stage_bytes), &map_w, (int)(f / kblocks) * kTileN,
+                            (int)(f % kblocks) * kSub, bar);
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            for (int it = 0; it < prefill; ++it)
+                tma_load_3d(s32(ring + (size_t)it * stage_bytes + a_bytes), &map_x, 0,
+                            (int)((f0 + it) % kblocks) * kSub, s32(&full[it]));
+            int it = prefill;
+            for (long long f = f0 + prefill; f < f1; ++f, ++it) {
                 const int t = (int)(f / kblocks), kb = (int)(f % kblocks);
                 const int s = it % p.stages;
-                if (it >= p.stages && !mbar_wait(s32(&empty[s]), ((it / p.stages) - 1) & 1)) { *failed = 1; break; }
+                if (!mbar_wait(s32(&empty[s]), ((it / p.stages) - 1) & 1)) { *failed = 1; break; }
                 if (*failed) break;
                 const uint32_t bar = s32(&full[s]);
                 uint8_t *st = ring + (size_t)s * stage_bytes;
@@ -285,6 +301,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const int et = threadIdx.x - 64;              // 0..127 among the epilogue threads
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // outputs, partials and tickets may still be in use
         int g = 0;
         for (long long f = f0; f < f1; ++g) {
             const int t = (int)(f / kblocks);
@@ -335,20 +352,20 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             if (*is_last) {
                 __threadfence();
                 const int cf_slot = (cut.first(cf) == start) ? 0 : 1;
-                // eight tokens at a time so that their loads are in flight together
-                for (int m0 = 0; m0 < p.M; m0 += 8) {
-                    float acc[8];
+                // sixteen tokens at a time so that their loads are in flight together
+                for (int m0 = 0; m0 < p.M; m0 += 16) {
+                    float acc[16];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+                    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
                     for (int c = 0; c < nc; ++c) {
                         const int sl = c == 0 ? 2 * cf + cf_slot : 2 * (cf + c);
                         const float *src = p.partials + ((size_t)sl * p.M + m0) * kTileN + et;
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
+                        for (int j = 0; j < 16; ++j)
                             if (m0 + j < p.M) acc[j] += __ldcg(src + (size_t)j * kTileN);
                     }
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
+                    for (int j = 0; j < 16; ++j)
                         if (m0 + j < p.M) store_out(p, m0 + j, t * kTileN + et, acc[j]);
                 }
             }
@@ -481,15 +498,26 @@ int isv_linear_forward(isv_linear *l, const void *x_dev, void *y_dev, float *y_f
     const size_t a_bytes = (size_t)kTileN * kTileK * 2, b_bytes = (size_t)p.mma_n * kTileK * 2;
     const size_t stage_bytes = a_bytes + ((b_bytes + 1023) & ~(size_t)1023);
     const size_t fixed = 1024 /* alignment slack */ + 1024 /* static */ + 512 /* barriers, slots */;
-    int stages = (int)std::min<size_t>(std::max<size_t>(3, (160u << 10) / stage_bytes), ((size_t)l->smem_optin - fixed) / stage_bytes);
+    // about 100 KB of ring: enough copies in flight, and the next launch's CTA fits beside this one's,
+    // so that its weight prefetch overlaps this launch's tail
+    int stages = (int)std::min<size_t>(std::max<size_t>(2, (100u << 10) / stage_bytes), ((size_t)l->smem_optin - fixed) / stage_bytes);
     if (stages < 2) return err(ISV_EINVAL, "shared memory too small for this batch");
     p.stages = stages;
     const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 4) * 8 + 64;
     CUtensorMap map_x;
     int rc = make_map(&map_x, x_dev, M, l->K, p.mma_n, l->bf16);   // rows beyond M read as zeros
     if (rc) return rc;
-    linear_kernel<<<l->grid, kThreads, smem, l->stream>>>(l->map_w, map_x, p);
-    cudaError_t e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(l->grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = l->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;   // see the kernel's griddepcontrol use
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_kernel, l->map_w, map_x, p);
     if (e != cudaSuccess) return err(ISV_ECUDA, "isv_linear_forward: %s", cudaGetErrorString(e));
     return ISV_OK;
 }
