@@ -98,6 +98,24 @@ class ShadowCache:
             self._k.setdefault((layer, s), []).append(k_bits[s][None].copy())
             self._v.setdefault((layer, s), []).append(v_bits[s][None].copy())
 
+    def store_at(self, layer: int, k_bits: np.ndarray, v_bits: np.ndarray, positions: Sequence[int]):
+        """Writes one token per sequence at explicit positions (overwriting what is there, or extending by
+        one).  This is what happens when several logical layers share one physical slab: each of them
+        writes its token of the step into the same slot, and the last writer's rows stay."""
+        assert k_bits.dtype == np.uint16 and v_bits.dtype == np.uint16
+        for s, pos in enumerate(positions):
+            k, v = self.gathered(layer, s)
+            assert 0 <= pos <= k.shape[0], "positions must overwrite or extend by one"
+            if pos == k.shape[0]:
+                k = np.concatenate([k, k_bits[s][None]])
+                v = np.concatenate([v, v_bits[s][None]])
+            else:
+                k = k.copy(); v = v.copy()
+                k[pos] = k_bits[s]
+                v[pos] = v_bits[s]
+            self._k[(layer, s)] = [k]
+            self._v[(layer, s)] = [v]
+
     def length(self, layer: int, s: int) -> int:
         return sum(c.shape[0] for c in self._k.get((layer, s), []))
 

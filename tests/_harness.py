@@ -41,6 +41,8 @@ class Harness:
         kw = B.desc_from_workload(w, **desc)
         kw["max_tokens_per_seq"] = max(kw["max_tokens_per_seq"], int(self.lens.max()) + w.steps)
         self.h = B.isv_kv_alloc(**kw)
+        # layers that share a physical slab share their record too (same order of writes)
+        self.phys = kw.get("phys_layers", 0) or w.layers
         self.shadow = km.ShadowCache(w.layers, w.kv_heads, w.head_dim)
         self.rng = W.host_rng(w)
         self.cur = self.lens.copy()
@@ -65,7 +67,7 @@ class Harness:
             kd, vd = bits_to_dev(k, w.dtype), bits_to_dev(v, w.dtype)
             torch.cuda.synchronize()
             B.isv_kv_fill(self.h, layer, kd, vd, self.lens, w.batch, T)
-            self.shadow.fill(layer, k, v, self.lens.tolist())
+            self.shadow.fill(layer % self.phys, k, v, self.lens.tolist())
 
     # ---- one decode step through separate append / attention calls
     def step(self, f32=True, out16=True, fused=False):
@@ -86,18 +88,27 @@ class Harness:
                 B.isv_kv_append(self.h, layer, kd, vd, w.batch)
                 B.isv_attn_decode(self.h, layer, qd, o16, of, None, None, w.batch)
             B.isv_sync(self.h)
-            self.shadow.append(layer, k, v)
-            res.append((q, of.cpu().numpy() if f32 else None, dev_to_bits(o16) if out16 else None))
+            if self.phys < w.layers:
+                # shared slabs: this layer's token lands at its own position, over a sharer's if one wrote first;
+                # the reference must be taken now, before the next sharer overwrites the slot again
+                self.shadow.store_at(layer % self.phys, k, v, self.cur.tolist())
+                ref = self.reference(layer, q, lens=(self.cur + 1))
+            else:
+                self.shadow.append(layer, k, v)
+                ref = None
+            res.append((q, of.cpu().numpy() if f32 else None, dev_to_bits(o16) if out16 else None, ref))
         self.cur += 1
         return res
 
     # ---- reference
-    def reference(self, layer: int, q_bits: np.ndarray, seqs=None) -> np.ndarray:
+    def reference(self, layer: int, q_bits: np.ndarray, seqs=None, lens=None) -> np.ndarray:
         w = self.w
         seqs = list(range(w.batch)) if seqs is None else list(seqs)
         K, V = [], []
         for s in seqs:
-            kb, vb = self.shadow.gathered(layer, s)
+            kb, vb = self.shadow.gathered(layer % self.phys, s)
+            if lens is not None:
+                kb, vb = kb[: int(lens[s])], vb[: int(lens[s])]
             K.append(values(kb, w.dtype))
             V.append(values(vb, w.dtype))
         q = values(q_bits[seqs], w.dtype)
@@ -107,8 +118,8 @@ class Harness:
         """Element-by-element comparison of one step's outputs with the reference."""
         w = self.w
         worst = 0.0
-        for layer, (q, of, o16) in enumerate(res):
-            ref = self.reference(layer, q)
+        for layer, (q, of, o16, ref_now) in enumerate(res):
+            ref = ref_now if ref_now is not None else self.reference(layer, q)
             if of is not None:
                 assert np.all(np.isfinite(of)), f"layer {layer}: non-finite output"
                 err = float(np.max(np.abs(of.astype(np.float64) - ref)))
@@ -126,7 +137,7 @@ class Harness:
         cap = B.isv_kv_info(self.h)
         for layer in (range(w.layers) if layers is None else layers):
             for s in (range(w.batch) if seqs is None else seqs):
-                kb, vb = self.shadow.gathered(layer, s)
+                kb, vb = self.shadow.gathered(layer % self.phys, s)
                 rows = max(1, kb.shape[0])
                 kh = np.zeros((rows, w.kv_heads, w.head_dim), np.uint16)
                 vh = np.zeros_like(kh)

@@ -115,6 +115,21 @@ def test_parity_over_head_grouping_head_dim_and_dtype(q_heads, kv_heads, head_di
         hz.check_gather()
 
 
+@pytest.mark.parametrize("f", [0.0, 0.5])
+@pytest.mark.parametrize("fused", [False, True])
+def test_layers_sharing_physical_slabs(f, fused):
+    """phys_layers < layers (how the benchmark fits 32-40 layers of a large batch): layers l and l + 2 write
+    the same slab, the later writer's rows stay; every layer's output is checked against the slab's content
+    at the time of its call, and the final slab content is read back bit for bit."""
+    lens = [5, 16, 31, 100, 48]
+    w = small(batch=len(lens), steps=20, f=f, perm=8, ctx=(1, 100), layers=4, q_heads=4, kv_heads=2, head_dim=64)
+    with Harness(w, lens=lens, phys_layers=2) as hz:
+        hz.fill()
+        for t in range(w.steps):
+            hz.check_step(hz.step(fused=fused))
+        hz.check_gather(layers=[2, 3])
+
+
 def test_identical_query_heads_of_a_group_give_identical_outputs():
     w = small(batch=2, steps=1, f=0.5, layers=1, q_heads=8, kv_heads=2, head_dim=128, ctx=(90, 90))
     with Harness(w) as hz:
@@ -141,7 +156,7 @@ def test_context_of_one_token_returns_v_exactly(f):
     with Harness(w, lens=[0, 0, 0]) as hz:
         hz.fill()
         res = hz.step()                                   # the appended token is the whole context
-        q, of, o16 = res[0]
+        q, of, o16, _ = res[0]
         kb, vb = zip(*[hz.shadow.gathered(0, s) for s in range(w.batch)])
         for s in range(w.batch):
             for h in range(w.q_heads):

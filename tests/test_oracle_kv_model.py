@@ -123,3 +123,17 @@ def test_shadow_cache_keeps_rows_in_arrival_order():
     gk, gv = sc.gathered(1, 2)
     assert np.array_equal(gk, k1[2][None]) and np.array_equal(gv, v1[2][None])
     assert sc.gathered(0, 0)[0].shape == (0, 2, 4)
+
+
+def test_shadow_cache_positional_store_overwrites_or_extends():
+    sc = km.ShadowCache(1, 1, 2)
+    a = np.array([[[1, 2]], [[3, 4]]], dtype=np.uint16)        # two sequences, one token each
+    sc.store_at(0, a, a + 10, [0, 0])                          # extend empty sequences
+    b = np.array([[[5, 6]], [[7, 8]]], dtype=np.uint16)
+    sc.store_at(0, b, b + 10, [0, 1])                          # overwrite seq 0's token, extend seq 1
+    k0, v0 = sc.gathered(0, 0)
+    k1, v1 = sc.gathered(0, 1)
+    assert k0.tolist() == [[[5, 6]]] and v0.tolist() == [[[15, 16]]]
+    assert k1.tolist() == [[[3, 4]], [[7, 8]]] and v1.tolist() == [[[13, 14]], [[17, 18]]]
+    with pytest.raises(AssertionError):
+        sc.store_at(0, b, b, [3, 0])
