@@ -103,6 +103,8 @@ struct isv_kv {
     int stages_res = 0, stages_stg = 0;
     size_t smem_res = 0, smem_stg = 0;
     uint64_t launches = 0;                 // kernels launched so far
+    int last_fused_layer = -1;             // layer of the latest fused decode launch if nothing else of ours
+                                           // was launched on the compute stream since, else -1
     // timing
     bool timing = false;
     std::vector<LayerEvents> lev;
@@ -217,6 +219,7 @@ int push_updates(isv_kv *h, const std::vector<TableUpdate> &upd) {
         }
         CU(launch_table_update(h->table_dev, b, h->s_compute));
         ++h->launches;
+        h->last_fused_layer = -1;
     }
     return ISV_OK;
 }
@@ -495,6 +498,7 @@ int isv_kv_reset(isv_kv *h) {
         CU(cudaMemset(h->tickets, 0, (size_t)h->g.max_seqs * h->g.Hkv * h->g.P * 4));
         std::fill(h->flush_recorded.begin(), h->flush_recorded.end(), 0);
         h->owner_uploaded = -1;
+        h->last_fused_layer = -1;
     }
     h->bm.reset();
     return ISV_OK;
@@ -560,6 +564,7 @@ int isv_kv_fill_async(isv_kv *h, int32_t layer, const void *k, const void *v, co
     const int pl = layer % g.phys_layers;
     if (h->flush_recorded[pl]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_flush[pl], 0));
     h->fill_timed = true;
+    h->last_fused_layer = -1;
     h->fill_stored = false;
     h->fill_bytes_stored = h->fill_bytes_resident = 0;
     h->fill_copies = 0;
@@ -706,6 +711,7 @@ int isv_kv_append(isv_kv *h, int32_t layer, const void *k, const void *v, int32_
     p.block_bytes = g.block_bytes;
     CU(launch_append(p, h->s_compute));
     ++h->launches;
+    h->last_fused_layer = -1;
     if (le) {
         CU(cudaEventRecord(le->a1, h->s_compute));
         le->have_append = true;
@@ -837,7 +843,10 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
             p.tail_w = h->tail ? h->tail + slab_tail(h, layer) : nullptr;
             // the kernel launched just before this one (the previous layer's, or a caller's) writes neither
             // the table, nor these lengths, nor this layer's slab: their reads need not wait for it
-            p.early_reads = (tables_settled && g.phys_layers > 1) ? 1 : 0;
+            // (it is the previous fused launch, of another layer on another slab, possibly followed by the
+            // caller's own kernels, which do not write library memory)
+            p.early_reads = (tables_settled && h->last_fused_layer >= 0 && h->last_fused_layer != layer &&
+                             h->last_fused_layer % g.phys_layers != layer % g.phys_layers) ? 1 : 0;
         }
         long long nu = 0;   // KV blocks in the flat work list
         for (int s = 0; s < n_seqs; ++s)
@@ -849,6 +858,7 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
         ++h->launches;
         if (le) CU(cudaEventRecord(le->r1, h->s_compute));
         if (k_new) h->lens_cur[layer] ^= 1;   // the kernel wrote the advanced lengths to the other copy
+        h->last_fused_layer = k_new ? layer : -1;
     }
 
     if (offloaded) {
@@ -985,6 +995,7 @@ int isv_kv_gather(isv_kv *h, int32_t layer, int32_t seq, void *k_host, void *v_h
     p.status = h->status_dev;
     p.seq = seq; p.len = n; p.n_pool_blocks = g.hbm_cap; p.n_host_blocks = g.host_cap;
     p.Hkv = g.Hkv; p.D = g.D; p.BT = g.BT; p.block_bytes = g.block_bytes;
+    h->last_fused_layer = -1;
     cudaError_t e = launch_gather(p, h->s_compute);
     ++h->launches;
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->s_compute);
