@@ -443,6 +443,7 @@ def main():
     ap.add_argument("--offload", type=float, default=None)
     ap.add_argument("--phys-layers", type=int, default=0)
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (small profiling cases)")
+    ap.add_argument("--batch", type=int, default=None, help="override the batch size (small profiling cases)")
     ap.add_argument("--zero-copy", action="store_true", help="read offloaded blocks in place instead of staging them")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -453,6 +454,8 @@ def main():
         w = w.with_(offload_frac=args.offload)
     if args.layers is not None:
         w = w.with_(layers=args.layers)
+    if args.batch is not None:
+        w = w.with_(batch=args.batch)
     if args.steps is None:
         args.steps = 128 if args.impl == "ours" and w.offload_frac == 0 else (5 if args.impl == "reference" else 4)
     if args.warmup < 0 or args.steps < 1:

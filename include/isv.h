@@ -55,7 +55,7 @@ extern "C" {
 #define ISV_BLOCK_NONE      (-1)
 #define ISV_BLOCK_HOST_BIT  (1 << 30)
 
-/* bits of the device status word (isv_step_times.status, isv_device_status) */
+/* bits of the device status word (isv_step_times.status, isv_sync, isv_linear_status) */
 #define ISV_STATUS_BAD_BLOCK_ID  1u   /* a table entry pointed outside its pool; block skipped */
 #define ISV_STATUS_WAIT_EXPIRED  2u   /* a bounded wait inside a kernel gave up                */
 
