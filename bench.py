@@ -37,9 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the resident decode kernel from one ncu capture (bytes per KV byte
 # processed), valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernels_sha1": "84b8539e1a4e25951c6fcbcecf757ffe7556feae",
-               # (546.95 MB read + 4.86 MB written) / 539.23 MB algorithmic, 2-layer case of the same shape
-               "dram_bytes_per_kv_byte": (546.951424 + 4.858880) / 539.230208,
+NCU_TRAFFIC = {"kernels_sha1": "a74bc63060974fddca0395cc5b4d8e50d2182e4e",
+               # (546.94 MB read + 4.76 MB written) / 539.23 MB algorithmic, 2-layer case of the same shape
+               "dram_bytes_per_kv_byte": (546.936832 + 4.763136) / 539.230208,
                "source": "profiles/decode_kernel_c2_2layers.md"}
 
 
