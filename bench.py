@@ -127,10 +127,11 @@ def reference_sample(w, ctx_lens, n_sample, rng):
     return q, K, V
 
 
-def time_reference(w, n_sample, reps, warmup=0):
+def time_reference(w, n_sample, reps, warmup=0, n_threads=0):
     """Times the CPU reference, as it stands, on a bounded sample: `n_sample`
-    sequences (all heads) of one layer-step.  Returns (tokens/s extrapolated to
-    the whole batch and all layers, seconds per sampled call, threads)."""
+    sequences (all heads) of one layer-step, on `n_threads` threads (0 = all the
+    process may use).  Returns (tokens/s extrapolated to the whole batch and all
+    layers, seconds per sampled call, threads, description of the sample)."""
     from oracle import attn as oa
     from paper_2504_11816_b200 import workloads as W
     lens = W.prompt_lens(w) + 1
@@ -142,7 +143,7 @@ def time_reference(w, n_sample, reps, warmup=0):
     times = []
     for i in range(warmup + reps):
         t0 = time.perf_counter()
-        oa.attn_decode(q, K, V)
+        oa.attn_decode(q, K, V, n_threads=n_threads)
         t1 = time.perf_counter()
         if i >= warmup:
             times.append(t1 - t0)
@@ -151,7 +152,7 @@ def time_reference(w, n_sample, reps, warmup=0):
     scale = float(lens.sum()) / float(ctx.sum())
     t_layer_step = t * scale
     tps = w.batch / (w.layers * t_layer_step)
-    return tps, t, oa.max_threads(), f"{n_sample} of {w.batch} sequences x {w.q_heads} heads, one layer-step " \
+    return tps, t, (n_threads or oa.max_threads()), f"{n_sample} of {w.batch} sequences x {w.q_heads} heads, one layer-step " \
         f"(contexts {int(ctx.min())}..{int(ctx.max())}), scaled by attended tokens to the batch and x{w.layers} layers"
 
 
@@ -414,10 +415,14 @@ def run_ours(args, w):
     # -------- CPU reference beside it (rank 0, single-GPU runs only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_sample = min(w.batch, 8 if w.name == "c2" else 4)
+        # C2: the whole batch, i.e. one full layer-step; the larger shapes: 4 sequences scaled up
+        n_sample = w.batch if w.name in ("c2", "tiny") else min(w.batch, 4)
         tps, t, threads, what = time_reference(w, n_sample, 3, 1)
+        tps1, t1_, _, what1 = time_reference(w, min(w.batch, 2), 1, 0, n_threads=1)
         cpu = {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what,
-               "seconds_per_sampled_call": t}
+               "seconds_per_sampled_call": t,
+               "one_thread": {"value": tps1, "unit": UNIT, "cores": 1, "sample": what1,
+                              "seconds_per_sampled_call": t1_}}
 
     if rank == 0:
         line = {

@@ -53,12 +53,15 @@ int oracle_attn_decode(const double *q, const double *K, const double *V,
     const int G = Hq / Hkv;
     const double inv_sqrt_d = 1.0 / sqrt((double)d);
     int failed = 0;
+    /* thread count for this call only (a global omp_set_num_threads would outlast it) */
+    int team = 1;
 #ifdef _OPENMP
-    if (n_threads > 0) omp_set_num_threads(n_threads);
+    team = n_threads > 0 ? n_threads : omp_get_max_threads();
 #else
     (void)n_threads;
+    (void)team;
 #endif
-#pragma omp parallel for schedule(dynamic, 1)
+#pragma omp parallel for schedule(dynamic, 1) num_threads(team)
     for (long sh = 0; sh < (long)n_seqs * Hq; ++sh) {
         const int s = (int)(sh / Hq);
         const int h = (int)(sh % Hq);
