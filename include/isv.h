@@ -22,7 +22,13 @@
  *     arithmetic is fp32.
  *   - KV pool layout, per physical layer and pool (HBM pool, host pool):
  *         [block][K|V][kv_head][block_tokens][head_dim]
- *     so one (block, K-or-V, head) tile is contiguous.
+ *     so one (block, K-or-V, head) tile is contiguous.  Inside a tile the row
+ *     of token t (head_dim elements) is stored as 16-byte chunks, and chunk c
+ *     sits at chunk position c XOR (t mod 8) of that row: the arrangement
+ *     that lets the tensor-core path load eight tokens at once without
+ *     shared-memory bank conflicts.  isv_kv_fill / isv_kv_append / isv_kv_gather
+ *     apply it; only a caller that builds a pool itself
+ *     (isv_attn_decode_static) has to.
  *   - Block table entry (int32): ISV_BLOCK_NONE = not allocated; otherwise the
  *     physical block id, with ISV_BLOCK_HOST_BIT set when the block belongs to
  *     the host pool.  The block that holds a sequence's newest token is kept in
@@ -315,7 +321,9 @@ int isv_linear_free(isv_linear *l);
  * cudaMalloc / cudaFree / cudaHostAlloc and uses no allocating library call;
  * it needs no handle.  The caller owns and passes every buffer:
  *   kv_pool_dev      KV pool in the library's layout,
- *                    [n_pool_blocks][K|V][kv_heads][block_tokens][head_dim], 16-bit
+ *                    [n_pool_blocks][K|V][kv_heads][block_tokens][head_dim], 16-bit,
+ *                    with the 16-byte chunks of each token row permuted as
+ *                    described under "KV pool layout" above
  *   block_table_dev  int32 [n_seqs][table_stride]: pool block ids in logical
  *                    order (ISV_BLOCK_NONE or host-flagged entries are skipped;
  *                    ids outside the pool are skipped and flagged)
@@ -329,10 +337,13 @@ int isv_linear_free(isv_linear *l);
  *   stream           cudaStream_t the work is enqueued on (asynchronous)
  * max_ctas: cap on the kernel's grid, 0 = one CTA per SM.
  * The split kernel's partial results and arrival counters live in one fixed
- * device array of ISV_STATIC_SCRATCH_BYTES.  A shape whose scratch
+ * device array of ISV_STATIC_SCRATCH_BYTES:
  *   n_seqs * (q_heads / heads per warp) * 4 B of counters
- *   + 2 * warps in the grid * heads per warp * (head_dim + 2) * 4 B of partials
- * does not fit is refused with ISV_ECAPACITY and a message; nothing runs then.
+ *   + 2 * warps in the grid * heads per warp * (head_dim + 2) * 4 B of partials.
+ * When the partials of a full grid do not fit, the grid is cut down to the
+ * CTAs whose partials do (the kernel divides the work among the CTAs it
+ * gets).  A shape that leaves no room for a single CTA is refused with
+ * ISV_ECAPACITY and a message; nothing runs then.
  * All calls on a GPU share that array and it keeps the previous call's
  * contents; each call zeroes the counters it needs on `stream` first.  Two
  * calls whose GPU work overlaps (different streams, or different threads

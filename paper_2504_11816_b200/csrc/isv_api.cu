@@ -758,7 +758,7 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
     base.table_stride = g.NB;
     base.q = q;
     base.status = h->status_dev;
-    base.n_seqs = n_seqs; base.Hq = g.Hq; base.Hkv = g.Hkv; base.P = g.P;
+    base.n_seqs = n_seqs; base.Hq = g.Hq; base.Hkv = g.Hkv; base.P = g.P; base.GT = g.GT;
     base.block_bytes = g.block_bytes;
     base.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)g.D));
 

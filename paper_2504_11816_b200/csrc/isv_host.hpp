@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "../../include/isv.h"
+#include "isv_kernels.cuh"
 
 namespace isv {
 
@@ -270,7 +271,7 @@ inline const char *make_geometry(const isv_kv_desc &d, Geometry *out) {
     g.Hq = d.q_heads;
     g.Hkv = d.kv_heads;
     g.G = g.Hq / g.Hkv;
-    g.GT = (g.G % 4 == 0) ? 4 : (g.G % 2 == 0) ? 2 : 1;
+    g.GT = group_heads(g.G);
     g.P = g.G / g.GT;
     if (d.head_dim != 64 && d.head_dim != 128) return "head_dim must be 64 or 128";
     g.D = d.head_dim;

@@ -117,6 +117,13 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
     }
 }
 
+// Inside a (block, K|V, head) tile the 16-byte chunk c of token t's row is stored at chunk position
+// c ^ (t & 7) of that row, in HBM, host memory and shared memory alike (tiles are copied verbatim).
+// Eight consecutive tokens then keep the same logical chunk in eight different bank groups, which makes
+// the matrix loads of the tensor-core path conflict-free; readers that take a whole 128-byte span of
+// one row per quarter-warp are unaffected.
+__device__ __forceinline__ int swz(int chunk, int t) { return chunk ^ (t & 7); }
+
 // ---------------------------------------------------------------- one K tile, one V tile
 
 // Lane layout inside a warp: grp = lane / 8 owns tokens grp, grp+4, ... of the
@@ -133,7 +140,7 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
 #pragma unroll
     for (int i = 0; i < NQ; ++i) {
         const int t = 4 * i + grp;
-        const uint4 *kp = reinterpret_cast<const uint4 *>(sK + t * ROW) + sub;
+        const uint4 *kp = reinterpret_cast<const uint4 *>(sK + t * ROW) + swz(sub, t);
         float a0[GT], a1[GT];   // two chains per dot product
 #pragma unroll
         for (int g = 0; g < GT; ++g) a0[g] = a1[g] = 0.f;
@@ -187,7 +194,7 @@ __device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp
                 pw[g] = exp2f(sc[i][g] - m[g]);
                 l[g] += pw[g];
             }
-            const uint4 *vp = reinterpret_cast<const uint4 *>(sV + t * ROW) + sub;
+            const uint4 *vp = reinterpret_cast<const uint4 *>(sV + t * ROW) + swz(sub, t);
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
                 float vf[8];
@@ -226,6 +233,453 @@ __device__ __forceinline__ void store_row_grouped(void *out, float *out_f32, siz
         }
     }
 }
+
+// ---------------------------------------------------------------- arithmetic of one warp
+//
+// The decode kernel is written once; what a warp does with a K tile, a V tile, this step's token and
+// its finished (m, l, o) state comes from one of two classes:
+//   ScalarMath  CUDA-core arithmetic, GT = 1 or 2 query heads per KV tile
+//   MmaMath     tensor-core arithmetic (mma.sync m16n8k16, fp32 accumulation) for grouped-query
+//               attention: the 3..16 query heads that share a KV head are the rows of one 16-row
+//               operand, so a KV tile is read once for all of them
+// Both keep scores in the log2 domain (the softmax scale is folded in with log2 e) and rescale the
+// accumulators lazily, only when a tile raises the running maximum.
+
+template <int D_, int GT_, int BT_, bool BF16_>
+struct ScalarMath {
+    static constexpr int D = D_, BT = BT_, E = D_ / 8;
+    static constexpr bool BF16 = BF16_;
+    float q[GT_][E], o[GT_][E], m[GT_], l[GT_], sc[BT_ / 4][GT_];
+    int grp, sub;
+
+    __device__ __forceinline__ void init(const DecodeParams &, int lane) {
+        grp = lane >> 3;
+        sub = lane & 7;
+    }
+    __device__ __forceinline__ int heads() const { return GT_; }
+
+    // New (sequence, head group): load its query rows (pre-scaled) and clear the state.
+    __device__ __forceinline__ void begin(const DecodeParams &p, int s, int hg) {
+#pragma unroll
+        for (int g = 0; g < GT_; ++g) {
+            const uint16_t *qrow =
+                reinterpret_cast<const uint16_t *>(p.q) + ((size_t)s * p.Hq + (size_t)hg * GT_ + g) * D;
+#pragma unroll
+            for (int v = 0; v < D / 64; ++v) {
+                const uint4 r = __ldg(reinterpret_cast<const uint4 *>(qrow + v * 64 + sub * 8));
+                float qf[8];
+                cvt8<BF16>(r, qf);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) q[g][v * 8 + e] = qf[e] * p.scale_log2;
+            }
+            m[g] = kNegBig;
+            l[g] = 0.f;
+#pragma unroll
+            for (int e = 0; e < E; ++e) o[g][e] = 0.f;
+        }
+    }
+    __device__ __forceinline__ void k_tile(const uint8_t *tile, int ntok) {
+        tile_scores<D, GT_, BT, BF16>(tile, ntok, grp, sub, q, sc, o, m, l);
+    }
+    __device__ __forceinline__ void v_tile(const uint8_t *tile, int ntok) {
+        tile_values<D, GT_, BT, BF16>(tile, ntok, grp, sub, sc, o, m, l);
+    }
+    // This step's token, read from the caller's rows: all groups compute its scores (the shuffles
+    // need every lane), group 0 keeps it.
+    __device__ __forceinline__ void new_token(const uint16_t *krow, const uint16_t *vrow) {
+        float a[GT_];
+#pragma unroll
+        for (int g = 0; g < GT_; ++g) a[g] = 0.f;
+#pragma unroll
+        for (int v = 0; v < D / 64; ++v) {
+            float kf[8];
+            cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(krow + v * 64 + sub * 8)), kf);
+#pragma unroll
+            for (int g = 0; g < GT_; ++g)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) a[g] = fmaf(q[g][v * 8 + e], kf[e], a[g]);
+        }
+#pragma unroll
+        for (int g = 0; g < GT_; ++g) {
+            a[g] += __shfl_xor_sync(kFull, a[g], 4);
+            a[g] += __shfl_xor_sync(kFull, a[g], 2);
+            a[g] += __shfl_xor_sync(kFull, a[g], 1);
+        }
+        if (grp == 0) {
+            float pw[GT_];
+#pragma unroll
+            for (int g = 0; g < GT_; ++g) {
+                if (a[g] > m[g]) {
+                    const float r = exp2f(m[g] - a[g]);
+                    l[g] *= r;
+#pragma unroll
+                    for (int e = 0; e < E; ++e) o[g][e] *= r;
+                    m[g] = a[g];
+                }
+                pw[g] = exp2f(a[g] - m[g]);
+                l[g] += pw[g];
+            }
+#pragma unroll
+            for (int v = 0; v < D / 64; ++v) {
+                float vf[8];
+                cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(vrow + v * 64 + sub * 8)), vf);
+#pragma unroll
+                for (int g = 0; g < GT_; ++g)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) o[g][v * 8 + e] = fmaf(pw[g], vf[e], o[g][v * 8 + e]);
+            }
+        }
+    }
+    // End of a unit: merge the four token groups of the warp (every group ends with the merged state).
+    __device__ __forceinline__ void finish() {
+#pragma unroll
+        for (int g = 0; g < GT_; ++g) {
+            float mm = fmaxf(m[g], __shfl_xor_sync(kFull, m[g], 8));
+            mm = fmaxf(mm, __shfl_xor_sync(kFull, mm, 16));
+            const float r = exp2f(m[g] - mm);
+            float ll = l[g] * r;
+            ll += __shfl_xor_sync(kFull, ll, 8);
+            ll += __shfl_xor_sync(kFull, ll, 16);
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                float x = o[g][e] * r;
+                x += __shfl_xor_sync(kFull, x, 8);
+                x += __shfl_xor_sync(kFull, x, 16);
+                o[g][e] = x;
+            }
+            m[g] = mm;
+            l[g] = ll;
+        }
+    }
+    // Folds the finished state into the running state of rows row0 .. row0 + GT - 1, which this
+    // unit alone writes in this launch.
+    __device__ __forceinline__ void fold_running(const DecodeParams &p, size_t row0) {
+#pragma unroll
+        for (int g = 0; g < GT_; ++g) {
+            const size_t row = row0 + g;
+            const float2 ml = *reinterpret_cast<const float2 *>(&p.acc_ml[row * 2]);
+            if (ml.y > 0.f) {
+                const float mm = fmaxf(m[g], ml.x);
+                const float a1 = exp2f(m[g] - mm), a2 = exp2f(ml.x - mm);
+                l[g] = l[g] * a1 + ml.y * a2;
+#pragma unroll
+                for (int v = 0; v < D / 64; ++v)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        o[g][v * 8 + e] = o[g][v * 8 + e] * a1 + p.acc_o[row * D + v * 64 + sub * 8 + e] * a2;
+                m[g] = mm;
+            }
+            __syncwarp();   // all lanes have read the old state before group 0 overwrites it
+            if (grp == 0) {
+                store_row_grouped<D, BF16>(nullptr, p.acc_o, row, sub, o[g], 1.f);
+                if (sub == 0) {
+                    p.acc_ml[row * 2] = m[g];
+                    p.acc_ml[row * 2 + 1] = l[g];
+                }
+            }
+        }
+    }
+    // Normalised result to out / out_f32, rows row0 .. row0 + GT - 1.
+    __device__ __forceinline__ void store_final(const DecodeParams &p, size_t row0) {
+        if (grp == 0) {
+#pragma unroll
+            for (int g = 0; g < GT_; ++g)
+                store_row_grouped<D, BF16>(p.out, p.out_f32, row0 + g, sub, o[g], l[g] > 0.f ? 1.f / l[g] : 0.f);
+        }
+    }
+    // Unnormalised (m, l, o) to rows row0 .. of o_dst / ml_dst (a partial slot or the resident result).
+    __device__ __forceinline__ void store_state(float *o_dst, float *ml_dst, size_t row0) {
+        if (grp == 0) {
+#pragma unroll
+            for (int g = 0; g < GT_; ++g) {
+                store_row_grouped<D, BF16>(nullptr, o_dst, row0 + g, sub, o[g], 1.f);
+                if (sub == 0) {
+                    ml_dst[(row0 + g) * 2] = m[g];
+                    ml_dst[(row0 + g) * 2 + 1] = l[g];
+                }
+            }
+        }
+    }
+};
+
+// D = A x B + D on one 16 x 8 tile, k = 16, 16-bit operands, fp32 accumulators.
+template <bool BF16>
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    if (BF16) {
+        asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    } else {
+        asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    }
+}
+// Four 8 x 8 matrices of 16-bit elements from shared memory; lane i gives the address of row i % 8 of
+// matrix i / 8 (16 bytes per row).  The transposing form hands out columns instead of rows.
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+template <bool BF16>
+__device__ __forceinline__ float2 unpack2(uint32_t w) {
+    if (BF16) return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    return __half22float2(*reinterpret_cast<const __half2 *>(&w));
+}
+
+// Tensor-core arithmetic for a group of 3..16 query heads that share one KV head (BT = 16).
+// Lane = 4 r + c.  Operand layouts of mma.m16n8k16 as used here:
+//   scores  S[head][token] = Q[head][dim] . K[token][dim]: A = Q (rows r and r + 8, held in registers
+//           for the whole segment), B = K read with ldmatrix (row = token, 8 dims per matrix row);
+//   output  O[head][dim] += P[head][token] . V[token][dim]: A = P, taken from the score accumulators
+//           (their layout is the A layout), B = V read with the transposing ldmatrix.
+// The weights P go to the tensor core as a 16-bit value plus a 16-bit remainder (two products per
+// V tile), so that rounding P to 16 bits does not limit the result's accuracy; l sums the fp32 weights.
+// Rows at or beyond the group's head count carry zero queries; their results are never stored.
+template <int D_, bool BF16_>
+struct MmaMath {
+    static constexpr int D = D_, BT = 16, ROW = D_ * 2;
+    static constexpr bool BF16 = BF16_;
+    uint32_t qa[D_ / 16][4];    // Q as A fragments, one per 16 dims
+    float oacc[D_ / 8][4];      // O accumulators: [j][0..1] row r, [j][2..3] row r + 8, dims 8 j + 2 c, + 1
+    float m[2], l[2];           // running maximum (same in the 4 lanes of a row) and this lane's share of the sum
+    uint32_t ph[4], pl[4];      // weights of the current block as A fragments: 16-bit value and remainder
+    float scale;
+    int lane, r, c, gt;
+
+    __device__ __forceinline__ void init(const DecodeParams &p, int lane_) {
+        lane = lane_;
+        r = lane_ >> 2;
+        c = lane_ & 3;
+        gt = p.GT;
+        scale = p.scale_log2;
+    }
+    __device__ __forceinline__ int heads() const { return gt; }
+
+    __device__ __forceinline__ void begin(const DecodeParams &p, int s, int hg) {
+        const uint16_t *qb = reinterpret_cast<const uint16_t *>(p.q) + ((size_t)s * p.Hq + (size_t)hg * gt) * D;
+        const uint32_t *q0 = reinterpret_cast<const uint32_t *>(qb + (size_t)r * D + 2 * c);
+        const uint32_t *q1 = reinterpret_cast<const uint32_t *>(qb + (size_t)(r + 8) * D + 2 * c);
+        const bool v0 = r < gt, v1 = r + 8 < gt;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+            qa[ks][0] = v0 ? __ldg(q0 + ks * 8) : 0u;
+            qa[ks][1] = v1 ? __ldg(q1 + ks * 8) : 0u;
+            qa[ks][2] = v0 ? __ldg(q0 + ks * 8 + 4) : 0u;
+            qa[ks][3] = v1 ? __ldg(q1 + ks * 8 + 4) : 0u;
+        }
+        m[0] = m[1] = kNegBig;
+        l[0] = l[1] = 0.f;
+#pragma unroll
+        for (int j = 0; j < D / 8; ++j) oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f;
+    }
+
+    // Raises the running maxima to (n0, n1) and rescales l and the accumulators accordingly.
+    __device__ __forceinline__ void raise_max(float n0, float n1) {
+        const float r0 = exp2f(m[0] - n0), r1 = exp2f(m[1] - n1);
+        l[0] *= r0;
+        l[1] *= r1;
+#pragma unroll
+        for (int j = 0; j < D / 8; ++j) {
+            oacc[j][0] *= r0;
+            oacc[j][1] *= r0;
+            oacc[j][2] *= r1;
+            oacc[j][3] *= r1;
+        }
+        m[0] = n0;
+        m[1] = n1;
+    }
+
+    __device__ __forceinline__ void k_tile(const uint8_t *tile, int ntok) {
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};   // tokens 0..7 and 8..15
+        const int tok = ((lane >> 4) << 3) + (lane & 7);
+        const uint32_t rowaddr = smem_u32(tile) + tok * ROW;
+        const int half = (lane >> 3) & 1;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4(rowaddr + (swz(2 * ks + half, tok) << 4), b0, b1, b2, b3);
+            mma16816<BF16>(s0, qa[ks], b0, b1);
+            mma16816<BF16>(s1, qa[ks], b2, b3);
+        }
+        // this lane's scores: rows r (x[0..3]) and r + 8 (y[0..3]) at tokens 2c, 2c+1, 2c+8, 2c+9
+        float x[4] = {s0[0] * scale, s0[1] * scale, s1[0] * scale, s1[1] * scale};
+        float y[4] = {s0[2] * scale, s0[3] * scale, s1[2] * scale, s1[3] * scale};
+        if (ntok < BT) {   // slots past the sequence end hold unspecified bits
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int t = 2 * c + (i & 1) + 8 * (i >> 1);
+                if (t >= ntok) x[i] = y[i] = kNegBig;
+            }
+        }
+        float mx0 = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+        float mx1 = fmaxf(fmaxf(y[0], y[1]), fmaxf(y[2], y[3]));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(kFull, mx0, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(kFull, mx1, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(kFull, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(kFull, mx1, 2));
+        if (__any_sync(kFull, mx0 > m[0] || mx1 > m[1])) raise_max(fmaxf(m[0], mx0), fmaxf(m[1], mx1));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            x[i] = exp2f(x[i] - m[0]);
+            y[i] = exp2f(y[i] - m[1]);
+        }
+        l[0] += (x[0] + x[1]) + (x[2] + x[3]);
+        l[1] += (y[0] + y[1]) + (y[2] + y[3]);
+        ph[0] = pack2<BF16>(x[0], x[1]);
+        ph[1] = pack2<BF16>(y[0], y[1]);
+        ph[2] = pack2<BF16>(x[2], x[3]);
+        ph[3] = pack2<BF16>(y[2], y[3]);
+        const float2 h0 = unpack2<BF16>(ph[0]), h1 = unpack2<BF16>(ph[1]);
+        const float2 h2 = unpack2<BF16>(ph[2]), h3 = unpack2<BF16>(ph[3]);
+        pl[0] = pack2<BF16>(x[0] - h0.x, x[1] - h0.y);
+        pl[1] = pack2<BF16>(y[0] - h1.x, y[1] - h1.y);
+        pl[2] = pack2<BF16>(x[2] - h2.x, x[3] - h2.y);
+        pl[3] = pack2<BF16>(y[2] - h3.x, y[3] - h3.y);
+    }
+
+    __device__ __forceinline__ void v_tile(const uint8_t *tile, int ntok) {
+        const int tok = (((lane >> 3) & 1) << 3) + (lane & 7);
+        const uint32_t rowaddr = smem_u32(tile) + tok * ROW;
+        const int hi = lane >> 4;
+        uint32_t k0 = 0xffffffffu, k1 = 0xffffffffu;   // keep-masks of the token pairs (2c, 2c+1) and (2c+8, 2c+9)
+        if (ntok < BT) {
+            k0 = (2 * c < ntok ? 0x0000ffffu : 0u) | (2 * c + 1 < ntok ? 0xffff0000u : 0u);
+            k1 = (2 * c + 8 < ntok ? 0x0000ffffu : 0u) | (2 * c + 9 < ntok ? 0xffff0000u : 0u);
+        }
+#pragma unroll
+        for (int jp = 0; jp < D / 16; ++jp) {
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4_t(rowaddr + (swz(2 * jp + hi, tok) << 4), b0, b1, b2, b3);
+            if (ntok < BT) {   // never let unspecified bits (possibly NaN patterns) reach a product
+                b0 &= k0; b1 &= k1; b2 &= k0; b3 &= k1;
+            }
+            mma16816<BF16>(oacc[2 * jp], ph, b0, b1);
+            mma16816<BF16>(oacc[2 * jp + 1], ph, b2, b3);
+            mma16816<BF16>(oacc[2 * jp], pl, b0, b1);
+            mma16816<BF16>(oacc[2 * jp + 1], pl, b2, b3);
+        }
+    }
+
+    // This step's token, read from the caller's rows, in plain fp32 arithmetic.
+    __device__ __forceinline__ void new_token(const uint16_t *krow, const uint16_t *vrow) {
+        float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+            const float2 ka = unpack2<BF16>(__ldg(reinterpret_cast<const uint32_t *>(krow + ks * 16 + 2 * c)));
+            const float2 kb = unpack2<BF16>(__ldg(reinterpret_cast<const uint32_t *>(krow + ks * 16 + 2 * c + 8)));
+            const float2 a0 = unpack2<BF16>(qa[ks][0]), a1 = unpack2<BF16>(qa[ks][1]);
+            const float2 a2 = unpack2<BF16>(qa[ks][2]), a3 = unpack2<BF16>(qa[ks][3]);
+            d0 = fmaf(a0.x, ka.x, d0); d0 = fmaf(a0.y, ka.y, d0); d0 = fmaf(a2.x, kb.x, d0); d0 = fmaf(a2.y, kb.y, d0);
+            d1 = fmaf(a1.x, ka.x, d1); d1 = fmaf(a1.y, ka.y, d1); d1 = fmaf(a3.x, kb.x, d1); d1 = fmaf(a3.y, kb.y, d1);
+        }
+        d0 += __shfl_xor_sync(kFull, d0, 1);
+        d1 += __shfl_xor_sync(kFull, d1, 1);
+        d0 += __shfl_xor_sync(kFull, d0, 2);
+        d1 += __shfl_xor_sync(kFull, d1, 2);
+        d0 *= scale;
+        d1 *= scale;
+        raise_max(fmaxf(m[0], d0), fmaxf(m[1], d1));
+        const float p0 = exp2f(d0 - m[0]), p1 = exp2f(d1 - m[1]);
+        if (c == 0) {   // l is summed over the 4 lanes of a row at the end: count the token once
+            l[0] += p0;
+            l[1] += p1;
+        }
+#pragma unroll
+        for (int j = 0; j < D / 8; ++j) {
+            const float2 v = unpack2<BF16>(__ldg(reinterpret_cast<const uint32_t *>(vrow + j * 8 + 2 * c)));
+            oacc[j][0] = fmaf(p0, v.x, oacc[j][0]);
+            oacc[j][1] = fmaf(p0, v.y, oacc[j][1]);
+            oacc[j][2] = fmaf(p1, v.x, oacc[j][2]);
+            oacc[j][3] = fmaf(p1, v.y, oacc[j][3]);
+        }
+    }
+
+    __device__ __forceinline__ void finish() {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            l[i] += __shfl_xor_sync(kFull, l[i], 1);
+            l[i] += __shfl_xor_sync(kFull, l[i], 2);
+        }
+    }
+
+    __device__ __forceinline__ void fold_running(const DecodeParams &p, size_t row0) {
+        float2 old[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int row = r + 8 * i;
+            old[i] = make_float2(kNegBig, 0.f);
+            if (row < gt) old[i] = *reinterpret_cast<const float2 *>(&p.acc_ml[(row0 + row) * 2]);
+        }
+        __syncwarp();   // the 4 lanes of a row have read (m, l) before lane c == 0 overwrites it
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int row = r + 8 * i;
+            if (row >= gt) continue;
+            float *orow = p.acc_o + (row0 + row) * D + 2 * c;
+            float a1 = 1.f, a2 = 0.f;
+            if (old[i].y > 0.f) {
+                const float mm = fmaxf(m[i], old[i].x);
+                a1 = exp2f(m[i] - mm);
+                a2 = exp2f(old[i].x - mm);
+                l[i] = l[i] * a1 + old[i].y * a2;
+                m[i] = mm;
+            }
+#pragma unroll
+            for (int j = 0; j < D / 8; ++j) {
+                float2 x = make_float2(oacc[j][2 * i] * a1, oacc[j][2 * i + 1] * a1);
+                if (old[i].y > 0.f) {
+                    const float2 y = *reinterpret_cast<const float2 *>(orow + j * 8);
+                    x.x = fmaf(y.x, a2, x.x);
+                    x.y = fmaf(y.y, a2, x.y);
+                }
+                *reinterpret_cast<float2 *>(orow + j * 8) = x;
+            }
+            if (c == 0) {
+                p.acc_ml[(row0 + row) * 2] = m[i];
+                p.acc_ml[(row0 + row) * 2 + 1] = l[i];
+            }
+        }
+    }
+
+    __device__ __forceinline__ void store_final(const DecodeParams &p, size_t row0) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int row = r + 8 * i;
+            if (row >= gt) continue;
+            const float inv = l[i] > 0.f ? 1.f / l[i] : 0.f;
+            const size_t idx = (row0 + row) * D + 2 * c;
+#pragma unroll
+            for (int j = 0; j < D / 8; ++j) {
+                const float x0 = oacc[j][2 * i] * inv, x1 = oacc[j][2 * i + 1] * inv;
+                if (p.out_f32) *reinterpret_cast<float2 *>(p.out_f32 + idx + j * 8) = make_float2(x0, x1);
+                if (p.out)
+                    *reinterpret_cast<uint32_t *>(reinterpret_cast<uint16_t *>(p.out) + idx + j * 8) =
+                        pack2<BF16>(x0, x1);
+            }
+        }
+    }
+
+    __device__ __forceinline__ void store_state(float *o_dst, float *ml_dst, size_t row0) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int row = r + 8 * i;
+            if (row >= gt) continue;
+            float *orow = o_dst + (row0 + row) * D + 2 * c;
+#pragma unroll
+            for (int j = 0; j < D / 8; ++j)
+                *reinterpret_cast<float2 *>(orow + j * 8) = make_float2(oacc[j][2 * i], oacc[j][2 * i + 1]);
+            if (c == 0) {
+                ml_dst[(row0 + row) * 2] = m[i];
+                ml_dst[(row0 + row) * 2 + 1] = l[i];
+            }
+        }
+    }
+};
 
 // Last-arriving contributor of a (sequence, head group): combine the nc partials of
 // query head g in fixed order.  Lane owns D/32 consecutive elements.
@@ -313,13 +767,16 @@ struct PendingArrival {
     size_t row0;
 };
 
-template <int D, int GT, int BT, bool BF16, int MODE, int NW>
+template <class Math, int MODE, int NW>
 __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p, const int stages) {
+    constexpr int D = Math::D, BT = Math::BT;
+    constexpr bool BF16 = Math::BF16;
     constexpr uint32_t TILE = BT * D * 2;
-    constexpr int E = D / 8;
     extern __shared__ __align__(128) uint8_t smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int grp = lane >> 3, sub = lane & 7;
+    Math mth;
+    mth.init(p, lane);
+    const int GT = mth.heads();   // query heads of one head group
 
     uint8_t *data = smem + (size_t)warp * stages * TILE;
     uint8_t *after_data = smem + (size_t)NW * stages * TILE;
@@ -584,7 +1041,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
                 if (lane < row_vecs) {
                     const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v_new : p.k_new) +
                                          ((size_t)s * p.Hkv + h) * (D * 2) + lane * 16;
-                    uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * TILE + (size_t)slot * (D * 2) + lane * 16;
+                    uint8_t *dst =
+                        base + (size_t)(kv * p.Hkv + h) * TILE + (size_t)slot * (D * 2) + swz(lane, slot) * 16;
                     *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
                 }
             } else if (lane == 0) {
@@ -614,7 +1072,6 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     };
 
     // ---- consumer
-    float q[GT][E], o[GT][E], m[GT], l[GT], sc[BT / 4][GT];
     int cur_seg = -1;
     int cons_stage = 0;
     uint32_t cons_phase = 0;
@@ -637,76 +1094,17 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         const int kind = flags & F_KIND_MASK;
         if (seg != cur_seg) {
             cur_seg = seg;
-#pragma unroll
-            for (int g = 0; g < GT; ++g) {
-                const uint16_t *qrow =
-                    reinterpret_cast<const uint16_t *>(p.q) + ((size_t)s * p.Hq + (size_t)hg * GT + g) * D;
-#pragma unroll
-                for (int v = 0; v < D / 64; ++v) {
-                    const uint4 r = __ldg(reinterpret_cast<const uint4 *>(qrow + v * 64 + sub * 8));
-                    float qf[8];
-                    cvt8<BF16>(r, qf);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) q[g][v * 8 + e] = qf[e] * p.scale_log2;
-                }
-                m[g] = kNegBig;
-                l[g] = 0.f;
-#pragma unroll
-                for (int e = 0; e < E; ++e) o[g][e] = 0.f;
-            }
+            mth.begin(p, s, hg);
         }
         const uint8_t *tile = data + (size_t)cons_stage * TILE;
         if (kind == F_KIND_K) {
-            tile_scores<D, GT, BT, BF16>(tile, ntok, grp, sub, q, sc, o, m, l);
+            mth.k_tile(tile, ntok);
         } else if (kind == F_KIND_V) {
-            tile_values<D, GT, BT, BF16>(tile, ntok, grp, sub, sc, o, m, l);
-        } else if (kind == F_KIND_NEW) {
-            // this step's token: all groups compute its scores (the shuffles need every lane), group 0 keeps it
+            mth.v_tile(tile, ntok);
+        } else if (kind == F_KIND_NEW) {   // this step's token, attended to from the caller's rows
             const int kvh = hg / p.P;
-            const uint16_t *krow = reinterpret_cast<const uint16_t *>(p.k_new) + ((size_t)s * p.Hkv + kvh) * D;
-            const uint16_t *vrow = reinterpret_cast<const uint16_t *>(p.v_new) + ((size_t)s * p.Hkv + kvh) * D;
-            float a[GT];
-#pragma unroll
-            for (int g = 0; g < GT; ++g) a[g] = 0.f;
-#pragma unroll
-            for (int v = 0; v < D / 64; ++v) {
-                float kf[8];
-                cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(krow + v * 64 + sub * 8)), kf);
-#pragma unroll
-                for (int g = 0; g < GT; ++g)
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) a[g] = fmaf(q[g][v * 8 + e], kf[e], a[g]);
-            }
-#pragma unroll
-            for (int g = 0; g < GT; ++g) {
-                a[g] += __shfl_xor_sync(kFull, a[g], 4);
-                a[g] += __shfl_xor_sync(kFull, a[g], 2);
-                a[g] += __shfl_xor_sync(kFull, a[g], 1);
-            }
-            if (grp == 0) {
-                float pw[GT];
-#pragma unroll
-                for (int g = 0; g < GT; ++g) {
-                    if (a[g] > m[g]) {
-                        const float r = exp2f(m[g] - a[g]);
-                        l[g] *= r;
-#pragma unroll
-                        for (int e = 0; e < E; ++e) o[g][e] *= r;
-                        m[g] = a[g];
-                    }
-                    pw[g] = exp2f(a[g] - m[g]);
-                    l[g] += pw[g];
-                }
-#pragma unroll
-                for (int v = 0; v < D / 64; ++v) {
-                    float vf[8];
-                    cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(vrow + v * 64 + sub * 8)), vf);
-#pragma unroll
-                    for (int g = 0; g < GT; ++g)
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) o[g][v * 8 + e] = fmaf(pw[g], vf[e], o[g][v * 8 + e]);
-                }
-            }
+            mth.new_token(reinterpret_cast<const uint16_t *>(p.k_new) + ((size_t)s * p.Hkv + kvh) * D,
+                          reinterpret_cast<const uint16_t *>(p.v_new) + ((size_t)s * p.Hkv + kvh) * D);
         }
         __syncwarp();   // every lane is done with this stage (data and metadata) before it is refilled
         --inflight;
@@ -716,95 +1114,31 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
 
         if (!(flags & F_LAST)) continue;
 
-        // ---- end of unit: merge the four token groups of the warp
-#pragma unroll
-        for (int g = 0; g < GT; ++g) {
-            float mm = fmaxf(m[g], __shfl_xor_sync(kFull, m[g], 8));
-            mm = fmaxf(mm, __shfl_xor_sync(kFull, mm, 16));
-            const float r = exp2f(m[g] - mm);
-            float ll = l[g] * r;
-            ll += __shfl_xor_sync(kFull, ll, 8);
-            ll += __shfl_xor_sync(kFull, ll, 16);
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                float x = o[g][e] * r;
-                x += __shfl_xor_sync(kFull, x, 8);
-                x += __shfl_xor_sync(kFull, x, 16);
-                o[g][e] = x;
-            }
-            m[g] = mm;
-            l[g] = ll;
-        }
+        // ---- end of unit
+        mth.finish();
+        const size_t row0 = (size_t)s * p.Hq + (size_t)hg * GT;
 
-        if (MODE == MODE_STAGED) {
-            // fold into the running state of (s, head); this unit is its only writer in this launch
-#pragma unroll
-            for (int g = 0; g < GT; ++g) {
-                const size_t row = (size_t)s * p.Hq + (size_t)hg * GT + g;
-                const float2 ml = *reinterpret_cast<const float2 *>(&p.acc_ml[row * 2]);
-                if (ml.y > 0.f) {
-                    const float mm = fmaxf(m[g], ml.x);
-                    const float a1 = exp2f(m[g] - mm), a2 = exp2f(ml.x - mm);
-                    l[g] = l[g] * a1 + ml.y * a2;
-#pragma unroll
-                    for (int v = 0; v < D / 64; ++v)
-#pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            o[g][v * 8 + e] =
-                                o[g][v * 8 + e] * a1 + p.acc_o[row * D + v * 64 + sub * 8 + e] * a2;
-                    m[g] = mm;
-                }
-                __syncwarp();   // all lanes have read the old state before group 0 overwrites it
-                if (grp == 0) {
-                    store_row_grouped<D, BF16>(nullptr, p.acc_o, row, sub, o[g], 1.f);
-                    if (sub == 0) {
-                        p.acc_ml[row * 2] = m[g];
-                        p.acc_ml[row * 2 + 1] = l[g];
-                    }
-                }
-            }
+        if (MODE == MODE_STAGED) {   // fold into the running state of (s, heads); this unit is its only writer
+            mth.fold_running(p, row0);
             continue;
         }
 
         // ---- resident mode
         if (nc == 1) {   // this warp covered the whole (sequence, head group): no partial needed
-            if (grp == 0) {
-#pragma unroll
-                for (int g = 0; g < GT; ++g) {
-                    const size_t row = (size_t)s * p.Hq + (size_t)hg * GT + g;
-                    if (p.finalize) {
-                        store_row_grouped<D, BF16>(p.out, p.out_f32, row, sub, o[g], l[g] > 0.f ? 1.f / l[g] : 0.f);
-                    } else {
-                        store_row_grouped<D, BF16>(nullptr, p.acc_o, row, sub, o[g], 1.f);
-                        if (sub == 0) {
-                            p.acc_ml[row * 2] = m[g];
-                            p.acc_ml[row * 2 + 1] = l[g];
-                        }
-                    }
-                }
-            }
+            if (p.finalize) mth.store_final(p, row0);
+            else mth.store_state(p.acc_o, p.acc_ml, row0);
             continue;
         }
         publish();   // the previous partial's arrival; its stores have long landed
         // an incomplete segment is the first or the last of its range: two partial slots per range
         const int slot = 2 * (mt_pack >> 2) + ((mt_pack & 2) ? 0 : 1);
-        if (grp == 0) {
-#pragma unroll
-            for (int g = 0; g < GT; ++g) {
-                const size_t pr = (size_t)slot * GT + g;
-                store_row_grouped<D, BF16>(nullptr, p.part_o, pr, sub, o[g], 1.f);
-                if (sub == 0) {
-                    p.part_ml[pr * 2] = m[g];
-                    p.part_ml[pr * 2 + 1] = l[g];
-                }
-            }
-        }
+        mth.store_state(p.part_o, p.part_ml, (size_t)slot * GT);
         pend.valid = 1;
         pend.ticket_idx = s * Hg + hg;
         pend.nc = nc;
         pend.wf = mt_wf;
         pend.wf_slot = mt_pack & 1;
-        pend.row0 = (size_t)s * p.Hq + (size_t)hg * GT;
+        pend.row0 = row0;
     }
     publish();
 }
@@ -878,7 +1212,8 @@ __global__ void append_kernel(const AppendParams p) {
             const int h = r / row_vecs, vec = r - h * row_vecs;
             const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
                                  ((size_t)s * p.Hkv + h) * row_bytes + vec * 16;
-            uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)slot * row_bytes + vec * 16;
+            uint8_t *dst =
+                base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)slot * row_bytes + swz(vec, slot) * 16;
             *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
         }
     } else if (threadIdx.x == 0) {
@@ -925,7 +1260,7 @@ __global__ void fill_kernel(const FillParams p) {
         const int t = r / row_vecs, vec = r - t * row_vecs;
         const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
                              (((size_t)s * p.T + (size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
-        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + vec * 16;
+        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + swz(vec, t) * 16;
         *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
     }
 }
@@ -945,7 +1280,7 @@ __global__ void pack_kernel(const PackParams p) {
         const int t = r / row_vecs, vec = r - t * row_vecs;
         const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
                              (((size_t)s * p.T + (size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
-        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + vec * 16;
+        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + swz(vec, t) * 16;
         *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
     }
 }
@@ -971,7 +1306,8 @@ __global__ void gather_kernel(const GatherParams p) {
         const int h = r / (ntok * row_vecs);
         r -= h * ntok * row_vecs;
         const int t = r / row_vecs, vec = r - t * row_vecs;
-        const uint8_t *src = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + vec * 16;
+        const uint8_t *src =
+            base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + swz(vec, t) * 16;
         uint8_t *dst = reinterpret_cast<uint8_t *>(kv ? p.v_out : p.k_out) +
                        (((size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
         *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
@@ -986,29 +1322,21 @@ __global__ void gather_kernel(const GatherParams p) {
 
 typedef void (*DecodeFn)(const DecodeParams, const int);
 
-template <int D, int GT, bool BF16>
+template <class Math, int NW>
 DecodeFn pick_mode(int mode) {
-    constexpr int NW = GT == 1 ? ISV_WARPS_GT1 : 8;
-    return mode == MODE_RESIDENT ? decode_kernel<D, GT, 16, BF16, MODE_RESIDENT, NW>
-                                 : decode_kernel<D, GT, 16, BF16, MODE_STAGED, NW>;
+    return mode == MODE_RESIDENT ? decode_kernel<Math, MODE_RESIDENT, NW> : decode_kernel<Math, MODE_STAGED, NW>;
 }
-template <int D, int GT>
-DecodeFn pick_dtype(bool bf16, int mode) {
-    return bf16 ? pick_mode<D, GT, true>(mode) : pick_mode<D, GT, false>(mode);
-}
-template <int D>
-DecodeFn pick_gt(int GT, bool bf16, int mode) {
-    switch (GT) {
-        case 1: return pick_dtype<D, 1>(bf16, mode);
-        case 2: return pick_dtype<D, 2>(bf16, mode);
-        case 4: return pick_dtype<D, 4>(bf16, mode);
-        default: return nullptr;
-    }
+template <int D, bool BF16>
+DecodeFn pick_gt(int GT, int mode) {
+    if (GT == 1) return pick_mode<ScalarMath<D, 1, 16, BF16>, ISV_WARPS_GT1>(mode);
+    if (GT == 2) return pick_mode<ScalarMath<D, 2, 16, BF16>, 8>(mode);
+    if (GT >= 3 && GT <= 16) return pick_mode<MmaMath<D, BF16>, 8>(mode);
+    return nullptr;
 }
 DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
     if (BT != 16) return nullptr;
-    if (D == 64) return pick_gt<64>(GT, bf16, mode);
-    if (D == 128) return pick_gt<128>(GT, bf16, mode);
+    if (D == 64) return bf16 ? pick_gt<64, true>(GT, mode) : pick_gt<64, false>(GT, mode);
+    if (D == 128) return bf16 ? pick_gt<128, true>(GT, mode) : pick_gt<128, false>(GT, mode);
     return nullptr;
 }
 

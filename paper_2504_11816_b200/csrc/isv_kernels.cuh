@@ -18,6 +18,8 @@ enum DecodeMode : int { MODE_RESIDENT = 0, MODE_STAGED = 1 };
 //     host-flagged newest block from its tail slot, skips other host blocks.
 //     A (sequence, head group) that spans several warps is finished by
 //     whichever of them arrives last (ticket), which merges their partials.
+//   A head group is GT query heads that share a KV head and are handled together on one KV tile:
+//     GT = 1 or 2 on the CUDA cores, 3..16 on the tensor cores (group_heads picks it).
 //   MODE_STAGED: units are (chunk unit, kv head x pass) from the plan lists;
 //     blocks are read from the staging buffer; results are merged into the
 //     running state acc_o / acc_ml, which one unit per launch owns.
@@ -53,6 +55,7 @@ struct DecodeParams {
     float *acc_ml;              // [n_seqs][Hq][2]
     uint32_t *status;
     int32_t n_seqs, Hq, Hkv, P;
+    int32_t GT;                 // query heads of one head group (Hq = Hkv * P * GT)
     int32_t finalize;           // resident: 1 = normalise and write out; 0 = leave (m, l, o) in acc_*
     int32_t early_reads;        // 1 = lengths, table and KV may be read before the dependency wait
     float scale_log2;           // log2(e) / sqrt(D)
@@ -117,6 +120,14 @@ struct MergeParams {
     float *out_f32;
     int32_t rows, D, bf16;
 };
+
+// Query heads handled together on one KV tile, for G query heads per KV head: the largest divisor of G
+// that is at most 16 (the row count of the tensor-core tile), so up to 16 heads read their KV once.
+inline int group_heads(int G) {
+    for (int gt = G < 16 ? G : 16; gt > 1; --gt)
+        if (G % gt == 0) return gt;
+    return 1;
+}
 
 // Warps per CTA of the decode kernel that handles GT query heads per KV tile.
 int decode_warps(int GT);

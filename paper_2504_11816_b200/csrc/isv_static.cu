@@ -82,7 +82,7 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     if (n_seqs == 0) return ISV_OK;
 
     const int G = q_heads / kv_heads;
-    const int GT = (G % 4 == 0) ? 4 : (G % 2 == 0) ? 2 : 1;
+    const int GT = group_heads(G);
     const int P = G / GT;
     if ((long long)n_seqs * max_blocks_per_seq * kv_heads * P >= (1ll << 31))
         return err(ISV_EINVAL, "isv_attn_decode_static: n_seqs * blocks * heads too large");
@@ -114,22 +114,28 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
         ds = g_dev[dev];
     }
 
-    // ---- scratch: counters per (sequence, head group) and two partials per warp of the grid
+    // ---- scratch: counters per (sequence, head group) and two partials per warp of the grid.
+    // A grid whose partials would not fit is cut down to the CTAs that do fit (the kernel is persistent
+    // and divides the work among however many CTAs it gets); only a shape that leaves no room for one
+    // CTA is refused.
     const int nw = decode_warps(GT);
     const long long blocks = (long long)n_seqs * max_blocks_per_seq * kv_heads * P;
     const int cap = max_ctas > 0 ? std::min(max_ctas, ds.sm_count) : ds.sm_count;
-    const int grid = (int)std::max<long long>(1, std::min<long long>(cap, (blocks + nw - 1) / nw));
-    const size_t slots = 2ull * grid * nw * GT;
+    int grid = (int)std::max<long long>(1, std::min<long long>(cap, (blocks + nw - 1) / nw));
     const size_t tickets_bytes = align256((size_t)n_seqs * kv_heads * P * 4);
-    const size_t ml_bytes = align256(slots * 2 * 4);
-    const size_t o_bytes = slots * head_dim * 4;
-    const size_t need = kHeaderBytes + tickets_bytes + ml_bytes + o_bytes;
-    if (need > (size_t)ISV_STATIC_SCRATCH_BYTES)
+    const size_t per_cta = 2ull * nw * GT * (2 + head_dim) * 4;   // (m, l) and o of two partials per warp and head
+    const size_t fixed = kHeaderBytes + tickets_bytes + 256;      // + alignment slack of the (m, l) array
+    const long long fit =
+        fixed < (size_t)ISV_STATIC_SCRATCH_BYTES ? (long long)(((size_t)ISV_STATIC_SCRATCH_BYTES - fixed) / per_cta) : 0;
+    if (fit < 1)
         return err(ISV_ECAPACITY,
                    "isv_attn_decode_static: this shape needs %lld bytes of scratch (arrival counters for %d sequences "
-                   "x %d head groups plus split partials) but the fixed array holds %lld; use fewer sequences or "
-                   "heads per call, a smaller max_ctas, or the handle-based isv_attn_decode",
-                   (long long)need, n_seqs, kv_heads * P, (long long)ISV_STATIC_SCRATCH_BYTES);
+                   "x %d head groups plus the split partials of one CTA) but the fixed array holds %lld; use fewer "
+                   "sequences or heads per call, or the handle-based isv_attn_decode",
+                   (long long)(fixed + per_cta), n_seqs, kv_heads * P, (long long)ISV_STATIC_SCRATCH_BYTES);
+    grid = (int)std::min<long long>(grid, fit);
+    const size_t slots = 2ull * grid * nw * GT;
+    const size_t ml_bytes = align256(slots * 2 * 4);
 
     // ---- shared-memory ring depth that fits
     const bool bf16 = dtype == ISV_BF16;
@@ -166,7 +172,7 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     p.part_o = reinterpret_cast<float *>(base + kHeaderBytes + tickets_bytes + ml_bytes);
     p.acc_o = nullptr;
     p.acc_ml = nullptr;
-    p.n_seqs = n_seqs; p.Hq = q_heads; p.Hkv = kv_heads; p.P = P;
+    p.n_seqs = n_seqs; p.Hq = q_heads; p.Hkv = kv_heads; p.P = P; p.GT = GT;
     p.finalize = 1;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)head_dim));
     p.block_bytes = 2ull * kv_heads * block_tokens * head_dim * 2ull;

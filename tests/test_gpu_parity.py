@@ -100,7 +100,10 @@ def test_result_does_not_depend_on_split_or_chunk_size(ctas, chunk_blocks):
 
 # ---------------------------------------------------------------- head grouping, head dim, dtype
 
-@pytest.mark.parametrize("q_heads,kv_heads", [(8, 8), (8, 4), (8, 2), (16, 2), (6, 2)])
+# query heads per KV head: 1 and 2 run on the CUDA cores, 3..16 as one tensor-core tile (4, 8, 3, 16, 12, 5),
+# 32 as two passes of 16
+@pytest.mark.parametrize("q_heads,kv_heads", [(8, 8), (8, 4), (8, 2), (16, 2), (6, 2), (32, 2), (24, 2), (10, 2),
+                                              (64, 2)])
 @pytest.mark.parametrize("head_dim", [64, 128])
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 def test_parity_over_head_grouping_head_dim_and_dtype(q_heads, kv_heads, head_dim, dtype):
@@ -151,8 +154,9 @@ def test_identical_query_heads_of_a_group_give_identical_outputs():
 # ---------------------------------------------------------------- special cases of the method
 
 @pytest.mark.parametrize("f", [0.0, 1.0])
-def test_context_of_one_token_returns_v_exactly(f):
-    w = small(batch=3, steps=1, f=f, layers=1, q_heads=4, kv_heads=2, head_dim=64, ctx=(0, 0))
+@pytest.mark.parametrize("q_heads", [4, 8])
+def test_context_of_one_token_returns_v_exactly(f, q_heads):
+    w = small(batch=3, steps=1, f=f, layers=1, q_heads=q_heads, kv_heads=2, head_dim=64, ctx=(0, 0))
     with Harness(w, lens=[0, 0, 0]) as hz:
         hz.fill()
         res = hz.step()                                   # the appended token is the whole context
@@ -160,12 +164,14 @@ def test_context_of_one_token_returns_v_exactly(f):
         kb, vb = zip(*[hz.shadow.gathered(0, s) for s in range(w.batch)])
         for s in range(w.batch):
             for h in range(w.q_heads):
-                assert np.array_equal(o16[s, h], vb[s][0, h // 2])
-                assert np.array_equal(of[s, h].astype(np.float64), oa.to_f64(values(vb[s][0, h // 2], w.dtype)))
+                g = h // (q_heads // 2)
+                assert np.array_equal(o16[s, h], vb[s][0, g])
+                assert np.array_equal(of[s, h].astype(np.float64), oa.to_f64(values(vb[s][0, g], w.dtype)))
 
 
-def test_zero_query_gives_the_mean_of_v():
-    w = small(batch=2, steps=1, f=0.5, layers=1, q_heads=4, kv_heads=4, head_dim=128, ctx=(333, 333))
+@pytest.mark.parametrize("q_heads", [4, 16])
+def test_zero_query_gives_the_mean_of_v(q_heads):
+    w = small(batch=2, steps=1, f=0.5, layers=1, q_heads=q_heads, kv_heads=4, head_dim=128, ctx=(333, 333))
     with Harness(w) as hz:
         hz.fill()
         k, v, q = W.host_step(w, hz.rng)
@@ -179,7 +185,8 @@ def test_zero_query_gives_the_mean_of_v():
         hz.shadow.append(0, k, v)
         for s in range(w.batch):
             vb = oa.to_f64(values(hz.shadow.gathered(0, s)[1], w.dtype))
-            assert np.max(np.abs(of[s].cpu().numpy() - vb.mean(axis=0))) <= 1e-5
+            mean = np.repeat(vb.mean(axis=0), q_heads // 4, axis=0)   # head h reads KV head h div (Hq / Hkv)
+            assert np.max(np.abs(of[s].cpu().numpy() - mean)) <= 1e-5
 
 
 def test_empty_sequences_yield_zeros_and_fewer_sequences_can_be_decoded():
@@ -205,10 +212,11 @@ def test_empty_sequences_yield_zeros_and_fewer_sequences_can_be_decoded():
         assert np.max(np.abs(o2[0] - ref[0])) <= TOL and np.all(o2[1:] == 7.0)
 
 
-def test_unused_slots_may_hold_nan_patterns():
+@pytest.mark.parametrize("q_heads", [4, 16])
+def test_unused_slots_may_hold_nan_patterns(q_heads):
     # fill every block with NaN bit patterns first, then reset and load short real data into the same blocks
     lens = [5, 21, 40]
-    w = small(batch=3, steps=4, f=0.5, layers=1, q_heads=4, kv_heads=4, head_dim=128, ctx=(1, 64))
+    w = small(batch=3, steps=4, f=0.5, layers=1, q_heads=q_heads, kv_heads=4, head_dim=128, ctx=(1, 64))
     with Harness(w, lens=lens) as hz:
         T = 64
         nan_bits = np.full((w.batch, T, w.kv_heads, w.head_dim), 0x7e00, np.uint16)

@@ -37,6 +37,13 @@ def _paged_pool(k_bits, v_bits, lens, kv_heads, head_dim, seed):
             t0, t1 = j * 16, min(int(lens[s]), j * 16 + 16)
             pool[bid, 0, :, : t1 - t0] = k_bits[s, t0:t1].transpose(1, 0, 2)
             pool[bid, 1, :, : t1 - t0] = v_bits[s, t0:t1].transpose(1, 0, 2)
+    # the documented chunk order inside a token row: 16-byte chunk c sits at position c ^ (t % 8)
+    chunks = pool.reshape(total, 2, kv_heads, 16, head_dim // 8, 8)
+    stored = np.empty_like(chunks)
+    for t in range(16):
+        for c in range(head_dim // 8):
+            stored[:, :, :, t, c ^ (t % 8)] = chunks[:, :, :, t, c]
+    pool = stored.reshape(total, 2, kv_heads, 16, head_dim)
     return pool, table, total, stride, max(nb)
 
 
@@ -88,8 +95,8 @@ def test_static_entry_matches_handle_entry_on_two_calls_in_a_row(q_heads, kv_hea
 def test_static_entry_refuses_shapes_beyond_its_fixed_scratch():
     one = torch.zeros(64, dtype=torch.int32, device="cuda")
     with pytest.raises(B.IsvError) as ei:
-        # 4096 sequences x 256 head groups: the arrival counters plus the partials exceed the fixed array
-        B.isv_attn_decode_static(one, 1, one, 64, one, 4096, 64, 1024, 256, 128, 16, B.ISV_F16, 0, one, one, None,
+        # 4096 sequences x 1024 head groups: the arrival counters alone exceed the fixed array
+        B.isv_attn_decode_static(one, 1, one, 64, one, 4096, 64, 1024, 1024, 128, 16, B.ISV_F16, 0, one, one, None,
                                  None, 0)
     assert ei.value.code == B.ISV_ECAPACITY
     assert "fixed array" in ei.value.message
