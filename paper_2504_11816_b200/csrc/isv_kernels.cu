@@ -745,9 +745,17 @@ __device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int wf
 
 // ---------------------------------------------------------------- decode kernel
 
-// Stage metadata words written by the producing lane before it arms the stage.
-enum { M_SEG = 0, M_SEQ, M_HG, M_NTOK, M_FLAGS, M_NC, M_WF, M_WFSLOT, M_WORDS = 8 };
-enum { F_KIND_K = 0, F_KIND_V = 1, F_KIND_END = 2, F_KIND_NEW = 3, F_KIND_MASK = 3, F_LAST = 4 };
+// A warp's work is a sequence of block visits.  A visit owns two slots of the warp's shared-memory
+// ring, one for the block's K tile and one for its V tile (each with its own mbarrier, so the scores
+// are computed while the V tile is still arriving), and one metadata record written by the producing
+// lane before it arms the K slot.  Visits without tiles (an empty unit, or a unit that consists of this
+// step's token only) arm both slots without a copy.
+enum { V_INFO = 0, V_SEQ, V_HG, V_NC, V_WF, V_PACK, V_WORDS = 8 };
+// V_INFO: bits 0..7 tokens in the block, then the flags
+enum { VF_DATA = 0x100,    // the visit has a K and a V tile
+       VF_FIRST = 0x200,   // first visit of a segment: load the queries, clear the state
+       VF_LAST = 0x400,    // last visit of a segment: store / fold / publish the state
+       VF_NEW = 0x800 };   // this step's token follows the block (fused append)
 
 // How the flat list of `total` work items is cut into `n` equal contiguous ranges, one per warp.
 // Ranges are numbered in item order, so the ranges that meet any interval are consecutive.
@@ -777,12 +785,13 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     Math mth;
     mth.init(p, lane);
     const int GT = mth.heads();   // query heads of one head group
+    const int NVIS = stages >> 1; // visits in flight per warp (stages is even)
 
     uint8_t *data = smem + (size_t)warp * stages * TILE;
     uint8_t *after_data = smem + (size_t)NW * stages * TILE;
     uint64_t *bars = reinterpret_cast<uint64_t *>(after_data) + warp * stages;
-    int32_t *meta = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * 8) + warp * stages * M_WORDS;
-    int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * (8 + 4 * M_WORDS));   // [n_seqs + 1]
+    int32_t *meta = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * 8) + warp * stages * V_WORDS;
+    int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * (8 + 4 * V_WORDS));   // [n_seqs + 1]
     int32_t *slen = ubase + p.n_seqs + 1;   // [n_seqs] tokens to attend (resident mode)
 
     // Programmatic dependent launch: let the next kernel in the stream begin its launch as this one's
@@ -797,6 +806,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
 
     const int Hg = p.Hkv * p.P;
     const uint64_t block_bytes = p.block_bytes;
+    const uint64_t v_off = (uint64_t)p.Hkv * TILE;   // from a block's K tile to its V tile of the same head
     const int fused = (MODE == MODE_RESIDENT && p.k_new != nullptr) ? 1 : 0;
 
     // ---- this warp's contiguous share of the work.  Resident mode: the flat space of KV blocks
@@ -846,18 +856,19 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     }
     __syncwarp();
 
-    // ---- producer state (identical in all lanes except `ent`)
-    int pu_seg = -1, pu_s = 0, pu_hg = 0, pu_nc = 1, pu_wf = 0, pu_wfslot = 0, pu_range = 0;
+    // ---- producer state (identical in all lanes except the two per-entry values)
+    int pu_s = 0, pu_hg = 0, pu_nc = 1, pu_wf = 0, pu_wfslot = 0;
     bool pu_first = true, range_first = true;   // the open segment is / the next one will be the first of its range
+    bool seg_start = false;                     // the next visit is the first of its segment
     int pu_len = 0, pu_jlast = -1, pu_j0 = 0, pu_n = 0;   // entries of the open unit: [pu_j0, pu_j0 + pu_n)
-    int pu_batch = 0, pu_nbatch = 0, pu_base = 0;
+    int pu_batch = 0, pu_nbatch = 0;
     uint32_t pu_mask = 0;
-    int32_t ent = ISV_BLOCK_NONE;
+    const uint8_t *ent_src = nullptr;   // lane i: K tile of entry i of the current batch of 32 entries
+    int ent_ntok = BT;                  // lane i: tokens of that block already in the cache, + 256 if it is the
+                                        // unit's newest block and this step's token follows it
     bool pu_open = false, pu_done = false;
-    const uint8_t *pv_src = nullptr;    // V tile of the block whose K tile was just issued
-    int pv_ntok = 0, pv_flags = 0;
-    int pn_flags = -1;                  // >= 0: a new-token stage is due after the current block
-    int prod_stage = 0, inflight = 0;
+    const uint8_t *pv_src = nullptr;    // V tile of the visit whose K slot was armed last (NULL: no tiles)
+    int prod_vis = 0, inflight = 0;     // ring position of the next visit to emit; visits emitted and not consumed
     if (MODE == MODE_RESIDENT) {   // sequence of the first unit: largest s with ubase[s] <= u_next
         int lo = 0, hi = p.n_seqs - 1;
         while (lo < hi) {
@@ -867,110 +878,73 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         pu_s = lo;
     }
 
-    auto emit = [&](const uint8_t *src, int ntok, int flags) {   // one stage: a tile, or a marker without data
-        if (lane == 0) {
-            int32_t *mt = meta + prod_stage * M_WORDS;
-            mt[M_SEG] = pu_seg; mt[M_SEQ] = pu_s; mt[M_HG] = pu_hg; mt[M_NTOK] = ntok; mt[M_FLAGS] = flags;
-            mt[M_NC] = pu_nc; mt[M_WF] = pu_wf;
-            mt[M_WFSLOT] = pu_wfslot | (pu_first ? 2 : 0) | (pu_range << 2);   // three fields in one word
-            const uint32_t bar = smem_u32(&bars[prod_stage]);
-            if (src) {
-                mbar_arrive_expect_tx(bar, TILE);
-                bulk_g2s(smem_u32(data + (size_t)prod_stage * TILE), src, TILE, bar);
-            } else {
-                mbar_arrive(bar);
-            }
-        }
-        prod_stage = (prod_stage + 1 == stages) ? 0 : prod_stage + 1;
-        ++inflight;
-    };
-
-    // Emits at most one stage.
-    auto produce = [&]() {
-        if (pv_src) {   // second half of the current block
-            emit(pv_src, pv_ntok, pv_flags);
-            pv_src = nullptr;
-            return;
-        }
-        if (pn_flags >= 0) {   // this step's token, read from the caller's k / v
-            emit(nullptr, 1, pn_flags);
-            pn_flags = -1;
-            return;
-        }
+    // Decides the next visit, writes its record and arms its K slot; the V slot is armed by produce_v
+    // (at once while the ring is being filled, later when the consumer has released that slot).
+    // Returns false when this warp's range is exhausted.
+    auto produce_k = [&]() -> bool {
+        int ntok = 0, flags = 0;
+        const uint8_t *ksrc = nullptr;
         while (true) {
             if (pu_mask != 0) {
                 const int i = __ffs(pu_mask) - 1;
                 pu_mask &= pu_mask - 1;
-                const int32_t e = __shfl_sync(kFull, ent, i);
+                const unsigned long long a = __shfl_sync(kFull, (unsigned long long)ent_src, i);
+                const int nt = __shfl_sync(kFull, ent_ntok, i);
                 const bool last = (pu_mask == 0) && (pu_batch >= pu_nbatch);
-                int ntok = BT;
-                const uint8_t *src;
-                if (MODE == MODE_RESIDENT) {
-                    const int j = pu_base + i;
-                    if (j == pu_jlast) ntok = pu_len - j * BT - fused;   // tokens already in the cache
-                    src = (e & ISV_BLOCK_HOST_BIT) ? p.tail + (uint64_t)pu_s * block_bytes
-                                                   : p.pool + (uint64_t)e * block_bytes;
-                    if (fused && j == pu_jlast) {
-                        if (last) pu_open = false;
-                        if (ntok == 0) {   // the new token opens this block
-                            emit(nullptr, 1, F_KIND_NEW | (last ? F_LAST : 0));
-                            return;
-                        }
-                        pn_flags = F_KIND_NEW | (last ? F_LAST : 0);
-                        const int kvh = pu_hg / p.P;
-                        pv_src = src + (uint64_t)(p.Hkv + kvh) * TILE;
-                        pv_ntok = ntok;
-                        pv_flags = F_KIND_V;
-                        emit(src + (uint64_t)kvh * TILE, ntok, F_KIND_K);
-                        return;
-                    }
-                } else {
-                    src = p.pool + (uint64_t)e * block_bytes;
+                ntok = nt & 255;
+                flags = (last ? VF_LAST : 0) | ((nt & 256) ? VF_NEW : 0);
+                if (ntok > 0) {
+                    flags |= VF_DATA;
+                    ksrc = reinterpret_cast<const uint8_t *>(a);
                 }
-                const int kvh = pu_hg / p.P;
-                pv_src = src + (uint64_t)(p.Hkv + kvh) * TILE;
-                pv_ntok = ntok;
-                pv_flags = F_KIND_V | (last ? F_LAST : 0);
-                emit(src + (uint64_t)kvh * TILE, ntok, F_KIND_K);
                 if (last) pu_open = false;
-                return;
+                break;
             }
             if (pu_open) {
-                if (pu_batch < pu_nbatch) {   // next 32 entries of the unit
-                    pu_base = pu_j0 + 32 * pu_batch;
+                if (pu_batch < pu_nbatch) {   // next 32 entries of the unit, one per lane
+                    const int j = pu_j0 + 32 * pu_batch + lane;
                     ++pu_batch;
-                    const int j = pu_base + lane;
                     bool valid = false;
-                    int32_t e = ISV_BLOCK_NONE;
+                    const uint8_t *src = nullptr;
+                    int nt = BT;
                     if (j < pu_j0 + pu_n) {
+                        int32_t e;
                         if (MODE == MODE_RESIDENT) {
                             e = p.table[(size_t)pu_s * p.table_stride + j];
                             if (e != ISV_BLOCK_NONE) {
-                                if (e & ISV_BLOCK_HOST_BIT) {
+                                if (e & ISV_BLOCK_HOST_BIT) {   // only the newest block of a sequence is read from its tail slot
                                     valid = (j == pu_jlast) && (p.tail != nullptr);
+                                    src = p.tail + (uint64_t)pu_s * block_bytes;
                                 } else {
                                     valid = e >= 0 && e < p.n_pool_blocks;
                                     if (!valid) atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+                                    src = p.pool + (uint64_t)e * block_bytes;
                                 }
                             }
+                            if (j == pu_jlast) nt = (pu_len - j * BT - fused) | (fused ? 256 : 0);
                         } else {
                             e = p.cblk[j];
                             valid = e >= 0 && e < p.n_pool_blocks;
                             if (!valid) atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+                            src = p.pool + (uint64_t)e * block_bytes;
                         }
                     }
-                    ent = e;
+                    ent_src = src + (uint64_t)(pu_hg / p.P) * TILE;
+                    ent_ntok = nt;
                     pu_mask = __ballot_sync(kFull, valid);
                     continue;
                 }
-                // no tile carried the end flag (or the unit is empty): explicit end marker
-                emit(nullptr, 0, F_KIND_END | F_LAST);
+                // no visit carried the end flag (or the unit is empty): explicit end marker
+                flags = VF_LAST;
                 pu_open = false;
-                return;
+                break;
             }
-            if (u_next >= u_end) { pu_done = true; return; }
+            if (u_next >= u_end) {
+                pu_done = true;
+                return false;
+            }
             // open the next segment (resident) or unit (staged)
-            ++pu_seg;
+            seg_start = true;
             if (MODE == MODE_RESIDENT) {
                 const int x = u_next;
                 while (x >= ubase[pu_s + 1]) ++pu_s;
@@ -986,7 +960,6 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
                 u_next = seg_end;
                 pu_n = nblk == 0 ? 0 : n;
                 pu_jlast = nblk - 1;
-                pu_range = cur_range;
                 pu_first = range_first;
                 range_first = false;
                 if (pu_j0 == 0 && n == nb) {
@@ -1011,9 +984,48 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             pu_mask = 0;
             pu_open = true;
         }
+        if (seg_start) {
+            flags |= VF_FIRST;
+            seg_start = false;
+        }
+        if (lane == 0) {
+            int32_t *mt = meta + prod_vis * V_WORDS;
+            mt[V_INFO] = ntok | flags;
+            mt[V_SEQ] = pu_s;
+            mt[V_HG] = pu_hg;
+            mt[V_NC] = pu_nc;
+            mt[V_WF] = pu_wf;
+            mt[V_PACK] = pu_wfslot | (pu_first ? 2 : 0) | (cur_range << 2);   // three fields in one word
+            const uint32_t bar = smem_u32(&bars[2 * prod_vis]);
+            if (ksrc) {
+                mbar_arrive_expect_tx(bar, TILE);
+                bulk_g2s(smem_u32(data + (size_t)(2 * prod_vis) * TILE), ksrc, TILE, bar);
+            } else {
+                mbar_arrive(bar);
+            }
+        }
+        pv_src = ksrc ? ksrc + v_off : nullptr;
+        ++inflight;
+        return true;
+    };
+    auto produce_v = [&]() {   // V slot of the visit produce_k emitted last; advances the ring position
+        if (lane == 0) {
+            const uint32_t bar = smem_u32(&bars[2 * prod_vis + 1]);
+            if (pv_src) {
+                mbar_arrive_expect_tx(bar, TILE);
+                bulk_g2s(smem_u32(data + (size_t)(2 * prod_vis + 1) * TILE), pv_src, TILE, bar);
+            } else {
+                mbar_arrive(bar);
+            }
+        }
+        prod_vis = (prod_vis + 1 == NVIS) ? 0 : prod_vis + 1;
     };
 
-    for (int i = 0; i < stages && !pu_done; ++i) produce();
+    if (!idle)
+        for (int i = 0; i < NVIS; ++i) {
+            if (!produce_k()) break;
+            produce_v();
+        }
     if (p.early_reads) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- fused append (placed after the first copies are in flight so that it costs no start-up time):
@@ -1052,7 +1064,6 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         }
     }
 
-
     // Publishes a stored partial: fence, ticket, and the merge if this was the last split to arrive.
     PendingArrival pend{0, 0, 0, 0, 0, 0};
     auto publish = [&]() {
@@ -1072,47 +1083,62 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     };
 
     // ---- consumer
-    int cur_seg = -1;
-    int cons_stage = 0;
+    int cons_vis = 0;
     uint32_t cons_phase = 0;
+    int s = 0, hg = 0;   // sequence and head group of the open segment
+    // A bounded wait ran out: report it, give the copies that may still be in flight one more bounded
+    // chance to land (slots of visit cons_vis onwards, in ring order), then leave.
+    auto give_up = [&]() {
+        if (lane == 0) atomicOr(p.status, ISV_STATUS_WAIT_EXPIRED);
+        for (int k = 0; k < inflight; ++k) {
+            mbar_wait(smem_u32(&bars[2 * cons_vis]), cons_phase);
+            mbar_wait(smem_u32(&bars[2 * cons_vis + 1]), cons_phase);
+            cons_vis = (cons_vis + 1 == NVIS) ? 0 : cons_vis + 1;
+            if (cons_vis == 0) cons_phase ^= 1u;
+        }
+    };
     while (inflight > 0) {
-        const bool ok = mbar_wait(smem_u32(&bars[cons_stage]), cons_phase);
+        bool ok = mbar_wait(smem_u32(&bars[2 * cons_vis]), cons_phase);
         if (!__all_sync(kFull, ok)) {
-            if (lane == 0) atomicOr(p.status, ISV_STATUS_WAIT_EXPIRED);
-            // give copies that may still be in flight one more bounded chance to land, then leave
-            for (int k = 0; k < inflight; ++k) {
-                mbar_wait(smem_u32(&bars[cons_stage]), cons_phase);
-                cons_stage = (cons_stage + 1 == stages) ? 0 : cons_stage + 1;
-                if (cons_stage == 0) cons_phase ^= 1u;
-            }
+            give_up();
             return;
         }
-        const int32_t *mt = meta + cons_stage * M_WORDS;
-        const int seg = mt[M_SEG], s = mt[M_SEQ], hg = mt[M_HG], nc = mt[M_NC];
-        const int ntok = mt[M_NTOK], flags = mt[M_FLAGS];
-        const int mt_wf = mt[M_WF], mt_pack = mt[M_WFSLOT];
-        const int kind = flags & F_KIND_MASK;
-        if (seg != cur_seg) {
-            cur_seg = seg;
+        const int32_t *mt = meta + cons_vis * V_WORDS;
+        const int info = mt[V_INFO];
+        const int ntok = info & 255;
+        int nc = 1, mt_wf = 0, mt_pack = 0;
+        if (info & VF_FIRST) {
+            s = mt[V_SEQ];
+            hg = mt[V_HG];
             mth.begin(p, s, hg);
         }
-        const uint8_t *tile = data + (size_t)cons_stage * TILE;
-        if (kind == F_KIND_K) {
-            mth.k_tile(tile, ntok);
-        } else if (kind == F_KIND_V) {
-            mth.v_tile(tile, ntok);
-        } else if (kind == F_KIND_NEW) {   // this step's token, attended to from the caller's rows
+        if (info & VF_LAST) {   // read now: the record is rewritten as soon as the K slot is handed back
+            nc = mt[V_NC];
+            mt_wf = mt[V_WF];
+            mt_pack = mt[V_PACK];
+        }
+        if (info & VF_DATA) mth.k_tile(data + (size_t)(2 * cons_vis) * TILE, ntok);
+        __syncwarp();   // every lane is done with the K slot and the record before they are refilled
+        const bool more = !pu_done && produce_k();
+
+        ok = mbar_wait(smem_u32(&bars[2 * cons_vis + 1]), cons_phase);
+        if (!__all_sync(kFull, ok)) {
+            give_up();
+            return;
+        }
+        if (info & VF_DATA) mth.v_tile(data + (size_t)(2 * cons_vis + 1) * TILE, ntok);
+        __syncwarp();   // every lane is done with the V slot before it is refilled
+        if (more) produce_v();
+        --inflight;
+        cons_vis = (cons_vis + 1 == NVIS) ? 0 : cons_vis + 1;
+        if (cons_vis == 0) cons_phase ^= 1u;
+
+        if (info & VF_NEW) {   // this step's token, attended to from the caller's rows
             const int kvh = hg / p.P;
             mth.new_token(reinterpret_cast<const uint16_t *>(p.k_new) + ((size_t)s * p.Hkv + kvh) * D,
                           reinterpret_cast<const uint16_t *>(p.v_new) + ((size_t)s * p.Hkv + kvh) * D);
         }
-        __syncwarp();   // every lane is done with this stage (data and metadata) before it is refilled
-        --inflight;
-        cons_stage = (cons_stage + 1 == stages) ? 0 : cons_stage + 1;
-        if (cons_stage == 0) cons_phase ^= 1u;
-        if (!pu_done) produce();
-
-        if (!(flags & F_LAST)) continue;
+        if (!(info & VF_LAST)) continue;
 
         // ---- end of unit
         mth.finish();
@@ -1320,6 +1346,10 @@ __global__ void gather_kernel(const GatherParams p) {
 #define ISV_WARPS_GT1 16   // warps per CTA when one query head is handled per KV tile
 #endif
 
+#ifndef ISV_WARPS_MMA
+#define ISV_WARPS_MMA 8   // warps per CTA of the tensor-core variant
+#endif
+
 typedef void (*DecodeFn)(const DecodeParams, const int);
 
 template <class Math, int NW>
@@ -1330,7 +1360,7 @@ template <int D, bool BF16>
 DecodeFn pick_gt(int GT, int mode) {
     if (GT == 1) return pick_mode<ScalarMath<D, 1, 16, BF16>, ISV_WARPS_GT1>(mode);
     if (GT == 2) return pick_mode<ScalarMath<D, 2, 16, BF16>, 8>(mode);
-    if (GT >= 3 && GT <= 16) return pick_mode<MmaMath<D, BF16>, 8>(mode);
+    if (GT >= 3 && GT <= 16) return pick_mode<MmaMath<D, BF16>, ISV_WARPS_MMA>(mode);
     return nullptr;
 }
 DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
@@ -1342,17 +1372,17 @@ DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
 
 }  // namespace
 
-int decode_warps(int GT) { return GT == 1 ? ISV_WARPS_GT1 : 8; }
+int decode_warps(int GT) { return GT == 1 ? ISV_WARPS_GT1 : GT == 2 ? 8 : ISV_WARPS_MMA; }
 
 int decode_default_stages(int D, int BT, int GT) {
     const int per_stage = decode_warps(GT) * BT * D * 2;
-    const int st = (128 << 10) / per_stage;
+    const int st = ((128 << 10) / per_stage) & ~1;   // slots come in pairs: a K and a V tile per block visit
     return st < 2 ? 2 : (st > 12 ? 12 : st);
 }
 
 size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode) {
     const size_t tile = (size_t)BT * D * 2;
-    size_t b = (size_t)decode_warps(GT) * stages * (tile + 8 + 4 * M_WORDS);
+    size_t b = (size_t)decode_warps(GT) * stages * (tile + 8 + 4 * V_WORDS);
     if (mode == MODE_RESIDENT) b += (size_t)(2 * max_seqs + 1) * 4;
     return b;
 }
@@ -1366,7 +1396,8 @@ cudaError_t decode_configure(int D, int GT, int BT, bool bf16, int mode, size_t 
 cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int BT, bool bf16, int mode, int grid,
                           int stages, size_t smem, cudaStream_t st) {
     DecodeFn fn = pick(D, GT, BT, bf16, mode);
-    if (!fn) return cudaErrorInvalidValue;
+    if (!fn || stages < 2) return cudaErrorInvalidValue;
+    stages &= ~1;   // the kernel uses its ring slots in pairs
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(decode_warps(GT) * 32);

@@ -132,8 +132,8 @@ inline int group_heads(int G) {
 // Warps per CTA of the decode kernel that handles GT query heads per KV tile.
 int decode_warps(int GT);
 
-// Ring depth per warp that keeps about 128 KiB of copies in flight per SM (measured on B200: deeper
-// rings lower the achieved HBM rate).
+// Ring depth per warp (tile slots, an even number: a block visit takes a K and a V slot) that keeps about
+// 128 KiB of copies in flight per SM (measured on B200: deeper rings lower the achieved HBM rate).
 int decode_default_stages(int D, int BT, int GT);
 
 // Bytes of dynamic shared memory the decode kernel needs for `stages` ring
