@@ -37,10 +37,15 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the resident decode kernel from one ncu capture (bytes per KV byte
 # processed), valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernels_sha1": "a74bc63060974fddca0395cc5b4d8e50d2182e4e",
-               # (546.94 MB read + 4.76 MB written) / 539.23 MB algorithmic, 2-layer case of the same shape
-               "dram_bytes_per_kv_byte": (546.936832 + 4.763136) / 539.230208,
-               "source": "profiles/decode_kernel_c2_2layers.md"}
+NCU_TRAFFIC = {"kernels_sha1": "fce0e5dc105aa2f9bb59af845bf8e516fa8fc232",
+               # multi-head shapes (CUDA-core arithmetic): (546.93 MB read + 4.46 MB written) / 539.23 MB
+               # algorithmic, 2-layer case of the default shape
+               "dram_bytes_per_kv_byte": (546.930432 + 4.460288) / 539.230208,
+               "source": "profiles/decode_kernel_c2_2layers.md",
+               # grouped-query shapes (tensor-core arithmetic): (540.01 MB + 5.85 MB) / 537.46 MB, 32 sequences
+               # and 2 layers of the 8B-GQA shape
+               "dram_bytes_per_kv_byte_gqa": (540.008960 + 5.848064) / 537.460736,
+               "source_gqa": "profiles/decode_kernel_gqa_c4shape_batch32_2layers.md"}
 
 
 def kernels_sha1() -> str:
@@ -350,8 +355,9 @@ def run_ours(args, w):
         timed = "separate pass of the same K steps with CUDA events around every launch"
     achieved = (bytes_res / n_launch) / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else 0.0
     traffic = None
-    if NCU_TRAFFIC["kernels_sha1"] == kernels_sha1() and NCU_TRAFFIC["dram_bytes_per_kv_byte"]:
-        traffic = NCU_TRAFFIC["dram_bytes_per_kv_byte"] * bytes_res / n_launch
+    if NCU_TRAFFIC["kernels_sha1"] == kernels_sha1():   # counters taken from this very kernel source
+        gqa = w.q_heads // w.kv_heads >= 3               # those shapes run the tensor-core variant
+        traffic = NCU_TRAFFIC["dram_bytes_per_kv_byte_gqa" if gqa else "dram_bytes_per_kv_byte"] * bytes_res / n_launch
     roofline = {"bound": "hbm", "kernel": "decode_kernel (resident, split flash-decoding)",
                 "achieved": achieved, "peak": hbm_gbs, "unit": "GB/s", "frac": achieved / hbm_gbs,
                 "peak_kind": f"of {peak_kind}", "traffic": traffic,

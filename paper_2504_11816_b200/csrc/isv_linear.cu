@@ -23,6 +23,7 @@
 #include <algorithm>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -500,7 +501,9 @@ int isv_linear_forward(isv_linear *l, const void *x_dev, void *y_dev, float *y_f
     const size_t fixed = 1024 /* alignment slack */ + 1024 /* static */ + 512 /* barriers, slots */;
     // about 100 KB of ring: enough copies in flight, and the next launch's CTA fits beside this one's,
     // so that its weight prefetch overlaps this launch's tail
-    int stages = (int)std::min<size_t>(std::max<size_t>(2, (100u << 10) / stage_bytes), ((size_t)l->smem_optin - fixed) / stage_bytes);
+    size_t ring_budget = 100u << 10;
+    if (const char *e = getenv("ISV_LINEAR_RING_KB")) ring_budget = (size_t)std::max(32, std::min(220, atoi(e))) << 10;   // tuning knob
+    int stages = (int)std::min<size_t>(std::max<size_t>(2, ring_budget / stage_bytes), ((size_t)l->smem_optin - fixed) / stage_bytes);
     if (stages < 2) return err(ISV_EINVAL, "shared memory too small for this batch");
     p.stages = stages;
     const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 4) * 8 + 64;
