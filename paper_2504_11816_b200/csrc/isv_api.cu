@@ -416,7 +416,7 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
     // scratch
     const size_t rows = (size_t)g.max_seqs * g.Hq;
     const int max_grid = g.max_ctas > 0 ? std::min(g.max_ctas, h->sm_count) : h->sm_count;
-    const size_t slots = 2ull * max_grid * decode_warps(g.GT) * g.GT;   // two partials per warp and query head
+    const size_t slots = 2ull * max_grid * decode_warps(g.GT, g.D) * g.GT;   // two partials per warp and query head
     if ((rc = dev_alloc((void **)&h->part_o, slots * g.D * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
     if ((rc = dev_alloc((void **)&h->part_ml, slots * 2 * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
     if ((rc = dev_alloc((void **)&h->tickets, (size_t)g.max_seqs * g.Hkv * g.P * 4, &h->scratch_bytes, "tickets"))) return bail(rc);
@@ -735,7 +735,7 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
     if (n_seqs == 0) return ISV_OK;
     const bool bf16 = g.dtype == ISV_BF16;
     const int Hg = g.Hkv * g.P;
-    const int nw = decode_warps(g.GT);
+    const int nw = decode_warps(g.GT, g.D);
     const OffPlan &pl = h->bm.plan(layer, n_seqs, h->zero_copy ? (1 << 30) : g.chunk_blocks);
     const bool offloaded = !pl.chunks.empty();
     const int phys = layer % g.phys_layers;

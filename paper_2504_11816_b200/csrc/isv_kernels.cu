@@ -238,9 +238,9 @@ __device__ __forceinline__ void store_row_grouped(void *out, float *out_f32, siz
 //
 // The decode kernel is written once; what a warp does with a K tile, a V tile, this step's token and
 // its finished (m, l, o) state comes from one of two classes:
-//   ScalarMath  CUDA-core arithmetic, GT = 1 or 2 query heads per KV tile
+//   ScalarMath  CUDA-core arithmetic, GT query heads per KV tile (used for GT = 1, multi-head attention)
 //   MmaMath     tensor-core arithmetic (mma.sync m16n8k16, fp32 accumulation) for grouped-query
-//               attention: the 3..16 query heads that share a KV head are the rows of one 16-row
+//               attention: the 2..16 query heads that share a KV head are the rows of one 16-row
 //               operand, so a KV tile is read once for all of them
 // Both keep scores in the log2 domain (the softmax scale is folded in with log2 e) and rescale the
 // accumulators lazily, only when a tile raises the running maximum.
@@ -431,7 +431,7 @@ __device__ __forceinline__ float2 unpack2(uint32_t w) {
     return __half22float2(*reinterpret_cast<const __half2 *>(&w));
 }
 
-// Tensor-core arithmetic for a group of 3..16 query heads that share one KV head (BT = 16).
+// Tensor-core arithmetic for a group of 2..16 query heads that share one KV head (BT = 16).
 // Lane = 4 r + c.  Operand layouts of mma.m16n8k16 as used here:
 //   scores  S[head][token] = Q[head][dim] . K[token][dim]: A = Q (rows r and r + 8, held in registers
 //           for the whole segment), B = K read with ldmatrix (row = token, 8 dims per matrix row);
@@ -1359,8 +1359,7 @@ DecodeFn pick_mode(int mode) {
 template <int D, bool BF16>
 DecodeFn pick_gt(int GT, int mode) {
     if (GT == 1) return pick_mode<ScalarMath<D, 1, 16, BF16>, ISV_WARPS_GT1>(mode);
-    if (GT == 2) return pick_mode<ScalarMath<D, 2, 16, BF16>, 8>(mode);
-    if (GT >= 3 && GT <= 16) return pick_mode<MmaMath<D, BF16>, ISV_WARPS_MMA>(mode);
+    if (GT >= 2 && GT <= 16) return pick_mode<MmaMath<D, BF16>, (D == 64 ? 16 : ISV_WARPS_MMA)>(mode);
     return nullptr;
 }
 DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
@@ -1372,17 +1371,19 @@ DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
 
 }  // namespace
 
-int decode_warps(int GT) { return GT == 1 ? ISV_WARPS_GT1 : GT == 2 ? 8 : ISV_WARPS_MMA; }
+// The tensor-core variant keeps 96 accumulator and operand registers per thread at head_dim 128 (8 warps);
+// at head_dim 64 it fits 128 registers, and 16 warps hide its per-visit latencies.
+int decode_warps(int GT, int D) { return GT == 1 ? ISV_WARPS_GT1 : (D == 64 ? 16 : ISV_WARPS_MMA); }
 
 int decode_default_stages(int D, int BT, int GT) {
-    const int per_stage = decode_warps(GT) * BT * D * 2;
+    const int per_stage = decode_warps(GT, D) * BT * D * 2;
     const int st = ((128 << 10) / per_stage) & ~1;   // slots come in pairs: a K and a V tile per block visit
     return st < 2 ? 2 : (st > 12 ? 12 : st);
 }
 
 size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode) {
     const size_t tile = (size_t)BT * D * 2;
-    size_t b = (size_t)decode_warps(GT) * stages * (tile + 8 + 4 * V_WORDS);
+    size_t b = (size_t)decode_warps(GT, D) * stages * (tile + 8 + 4 * V_WORDS);
     if (mode == MODE_RESIDENT) b += (size_t)(2 * max_seqs + 1) * 4;
     return b;
 }
@@ -1400,7 +1401,7 @@ cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int BT, bool bf1
     stages &= ~1;   // the kernel uses its ring slots in pairs
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(decode_warps(GT) * 32);
+    cfg.blockDim = dim3(decode_warps(GT, D) * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

@@ -19,7 +19,7 @@ enum DecodeMode : int { MODE_RESIDENT = 0, MODE_STAGED = 1 };
 //     A (sequence, head group) that spans several warps is finished by
 //     whichever of them arrives last (ticket), which merges their partials.
 //   A head group is GT query heads that share a KV head and are handled together on one KV tile:
-//     GT = 1 or 2 on the CUDA cores, 3..16 on the tensor cores (group_heads picks it).
+//     GT = 1 on the CUDA cores, 2..16 on the tensor cores (group_heads picks it).
 //   MODE_STAGED: units are (chunk unit, kv head x pass) from the plan lists;
 //     blocks are read from the staging buffer; results are merged into the
 //     running state acc_o / acc_ml, which one unit per launch owns.
@@ -129,8 +129,8 @@ inline int group_heads(int G) {
     return 1;
 }
 
-// Warps per CTA of the decode kernel that handles GT query heads per KV tile.
-int decode_warps(int GT);
+// Warps per CTA of the decode kernel that handles GT query heads per KV tile at head_dim D.
+int decode_warps(int GT, int D);
 
 // Ring depth per warp (tile slots, an even number: a block visit takes a K and a V slot) that keeps about
 // 128 KiB of copies in flight per SM (measured on B200: deeper rings lower the achieved HBM rate).

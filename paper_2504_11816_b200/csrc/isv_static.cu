@@ -118,7 +118,7 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     // A grid whose partials would not fit is cut down to the CTAs that do fit (the kernel is persistent
     // and divides the work among however many CTAs it gets); only a shape that leaves no room for one
     // CTA is refused.
-    const int nw = decode_warps(GT);
+    const int nw = decode_warps(GT, head_dim);
     const long long blocks = (long long)n_seqs * max_blocks_per_seq * kv_heads * P;
     const int cap = max_ctas > 0 ? std::min(max_ctas, ds.sm_count) : ds.sm_count;
     int grid = (int)std::max<long long>(1, std::min<long long>(cap, (blocks + nw - 1) / nw));
