@@ -743,6 +743,91 @@ __device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int wf
     }
 }
 
+// The same combination for R query heads of the group at once (g0 .. g0 + R - 1, those below GT): the
+// loads of all R rows of a contributor are in flight together, so a group of many heads costs a few memory
+// round trips instead of a few per head.  Used where the warp's accumulators are no longer live (at the end
+// of its range); per head the arithmetic and its order are those of merge_partials_row.
+template <int D, bool BF16, int R>
+__device__ __forceinline__ void merge_partials_rows(const DecodeParams &p, int wf, int wf_slot, int nc, int g0, int GT,
+                                                    size_t row0, int lane) {
+    constexpr int EPL = D / 32;
+    auto slot_of = [&](int c) { return c == 0 ? 2 * wf + wf_slot : 2 * (wf + c); };
+    float mm[R], ll[R], acc[R][EPL];
+#pragma unroll
+    for (int j = 0; j < R; ++j) {
+        mm[j] = kNegBig;
+        ll[j] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[j][e] = 0.f;
+    }
+    for (int c = 0; c < nc; ++c) {   // every lane reads the same words: broadcast loads
+        const float *ml = p.part_ml + ((size_t)slot_of(c) * GT + g0) * 2;
+#pragma unroll
+        for (int j = 0; j < R; ++j)
+            if (g0 + j < GT) mm[j] = fmaxf(mm[j], __ldcg(ml + 2 * j));
+    }
+    for (int c = 0; c < nc; ++c) {
+        const size_t pr = (size_t)slot_of(c) * GT + g0;
+        float2 ml[R];
+        float x[R][EPL];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            ml[j] = make_float2(kNegBig, 0.f);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) x[j][e] = 0.f;
+            if (g0 + j < GT) {
+                ml[j] = __ldcg(reinterpret_cast<const float2 *>(&p.part_ml[(pr + j) * 2]));
+                const float *po = p.part_o + (pr + j) * D + lane * EPL;
+                if (EPL == 4) {
+                    const float4 v = __ldcg(reinterpret_cast<const float4 *>(po));
+                    x[j][0] = v.x; x[j][1] = v.y; x[j][2] = v.z; x[j][3] = v.w;
+                } else {
+                    const float2 v = __ldcg(reinterpret_cast<const float2 *>(po));
+                    x[j][0] = v.x; x[j][1] = v.y;
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            const float a = exp2f(ml[j].x - mm[j]);
+            ll[j] += ml[j].y * a;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) acc[j][e] = fmaf(a, x[j][e], acc[j][e]);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < R; ++j) {
+        if (g0 + j >= GT) continue;
+        const size_t row = row0 + g0 + j;
+        const size_t idx = row * D + lane * EPL;
+        if (p.finalize) {
+            const float inv = ll[j] > 0.f ? 1.f / ll[j] : 0.f;
+            if (p.out_f32) {
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) p.out_f32[idx + e] = acc[j][e] * inv;
+            }
+            if (p.out) {
+                uint16_t *o16 = reinterpret_cast<uint16_t *>(p.out) + idx;
+                if (EPL == 4) {
+                    uint2 w;
+                    w.x = pack2<BF16>(acc[j][0] * inv, acc[j][1] * inv);
+                    w.y = pack2<BF16>(acc[j][2] * inv, acc[j][3] * inv);
+                    *reinterpret_cast<uint2 *>(o16) = w;
+                } else {
+                    *reinterpret_cast<uint32_t *>(o16) = pack2<BF16>(acc[j][0] * inv, acc[j][1] * inv);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) p.acc_o[idx + e] = acc[j][e];
+            if (lane == 0) {
+                p.acc_ml[row * 2] = mm[j];
+                p.acc_ml[row * 2 + 1] = ll[j];
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------- decode kernel
 
 // A warp's work is a sequence of block visits.  A visit owns two slots of the warp's shared-memory
@@ -1066,7 +1151,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
 
     // Publishes a stored partial: fence, ticket, and the merge if this was the last split to arrive.
     PendingArrival pend{0, 0, 0, 0, 0, 0};
-    auto publish = [&]() {
+    auto publish = [&](bool at_end) {
         if (!pend.valid) return;
         pend.valid = 0;
         __syncwarp();   // the lanes' partial stores are ordered before lane 0's release below
@@ -1077,8 +1162,13 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         ticket = __shfl_sync(kFull, ticket, 0);   // the other lanes read the partials after lane 0's acquire
         if (ticket == pend.nc - 1) {
             if (lane == 0) p.tickets[pend.ticket_idx] = 0;   // ready for the next launch
-            for (int g = 0; g < GT; ++g)
-                merge_partials_row<D, BF16>(p, pend.wf, pend.wf_slot, pend.nc, g, GT, pend.row0 + g, lane);
+            if (at_end && GT > 1) {   // the accumulators are dead: several heads at a time
+                for (int g0 = 0; g0 < GT; g0 += 8)
+                    merge_partials_rows<D, BF16, 8>(p, pend.wf, pend.wf_slot, pend.nc, g0, GT, pend.row0, lane);
+            } else {
+                for (int g = 0; g < GT; ++g)
+                    merge_partials_row<D, BF16>(p, pend.wf, pend.wf_slot, pend.nc, g, GT, pend.row0 + g, lane);
+            }
         }
     };
 
@@ -1155,7 +1245,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             else mth.store_state(p.acc_o, p.acc_ml, row0);
             continue;
         }
-        publish();   // the previous partial's arrival; its stores have long landed
+        publish(false);   // the previous partial's arrival; its stores have long landed
         // an incomplete segment is the first or the last of its range: two partial slots per range
         const int slot = 2 * (mt_pack >> 2) + ((mt_pack & 2) ? 0 : 1);
         mth.store_state(p.part_o, p.part_ml, (size_t)slot * GT);
@@ -1166,7 +1256,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         pend.wf_slot = mt_pack & 1;
         pend.row0 = row0;
     }
-    publish();
+    publish(true);
 }
 
 // ---------------------------------------------------------------- merge kernel (resident + offloaded)
