@@ -24,7 +24,8 @@
  *         [block][K|V][kv_head][block_tokens][head_dim]
  *     so one (block, K-or-V, head) tile is contiguous.  Inside a tile the row
  *     of token t (head_dim elements) is stored as 16-byte chunks, and chunk c
- *     sits at chunk position c XOR (t mod 8) of that row: the arrangement
+ *     sits at chunk position c XOR (t mod 8) of that row (head_dim 80: chunks
+ *     0..7 only; chunks 8 and 9 stay in place): the arrangement
  *     that lets the tensor-core path load eight tokens at once without
  *     shared-memory bank conflicts.  isv_kv_fill / isv_kv_append / isv_kv_gather
  *     apply it; only a caller that builds a pool itself
@@ -78,7 +79,7 @@ typedef struct {
                                  /* layers; layers sharing a slab overwrite each other's data)  */
     int32_t  q_heads;            /* query heads; multiple of kv_heads                           */
     int32_t  kv_heads;
-    int32_t  head_dim;           /* 64 or 128                                                   */
+    int32_t  head_dim;           /* 64, 80 (OPT-2.7B, the paper's main model: h1 2560 / 32) or 128 */
     int32_t  block_tokens;       /* tokens per KV block; 16                                     */
     int32_t  dtype;              /* ISV_F16 or ISV_BF16                                         */
     float    offload_frac;       /* C_off in [0, 1]: of every prefix of j blocks of a sequence, */

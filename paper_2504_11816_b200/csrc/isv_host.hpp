@@ -273,7 +273,7 @@ inline const char *make_geometry(const isv_kv_desc &d, Geometry *out) {
     g.G = g.Hq / g.Hkv;
     g.GT = group_heads(g.G);
     g.P = g.G / g.GT;
-    if (d.head_dim != 64 && d.head_dim != 128) return "head_dim must be 64 or 128";
+    if (d.head_dim != 64 && d.head_dim != 80 && d.head_dim != 128) return "head_dim must be 64, 80 or 128";
     g.D = d.head_dim;
     if (d.block_tokens != 16) return "block_tokens must be 16";
     g.BT = d.block_tokens;

@@ -121,8 +121,11 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 // c ^ (t & 7) of that row, in HBM, host memory and shared memory alike (tiles are copied verbatim).
 // Eight consecutive tokens then keep the same logical chunk in eight different bank groups, which makes
 // the matrix loads of the tensor-core path conflict-free; readers that take a whole 128-byte span of
-// one row per quarter-warp are unaffected.
-__device__ __forceinline__ int swz(int chunk, int t) { return chunk ^ (t & 7); }
+// one row per quarter-warp are unaffected.  A row of `nchunks` chunks is permuted in its complete groups
+// of eight; a trailing incomplete group (head_dim 80: chunks 8 and 9) stays in place.
+__device__ __forceinline__ int swz(int chunk, int t, int nchunks) {
+    return chunk < (nchunks & ~7) ? chunk ^ (t & 7) : chunk;
+}
 
 // ---------------------------------------------------------------- one K tile, one V tile
 
@@ -134,20 +137,21 @@ __device__ __forceinline__ int swz(int chunk, int t) { return chunk ^ (t & 7); }
 // pre-scaled), and the running maximum brought up to date (o and l rescaled).
 template <int D, int GT, int BT, bool BF16>
 __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp, int sub,
-                                            const float (&q)[GT][D / 8], float (&sc)[BT / 4][GT],
-                                            float (&o)[GT][D / 8], float (&m)[GT], float (&l)[GT]) {
-    constexpr int NV = D / 64, NQ = BT / 4, ROW = D * 2;
+                                            const float (&q)[GT][(D + 63) / 64 * 8], float (&sc)[BT / 4][GT],
+                                            float (&o)[GT][(D + 63) / 64 * 8], float (&m)[GT], float (&l)[GT]) {
+    constexpr int NV = (D + 63) / 64, NQ = BT / 4, ROW = D * 2;
 #pragma unroll
     for (int i = 0; i < NQ; ++i) {
         const int t = 4 * i + grp;
-        const uint4 *kp = reinterpret_cast<const uint4 *>(sK + t * ROW) + swz(sub, t);
+        const uint4 *krow = reinterpret_cast<const uint4 *>(sK + t * ROW);
         float a0[GT], a1[GT];   // two chains per dot product
 #pragma unroll
         for (int g = 0; g < GT; ++g) a0[g] = a1[g] = 0.f;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
+            if ((v + 1) * 64 > D && v * 64 + sub * 8 >= D) continue;   // last, incomplete 64-element span
             float kf[8];
-            cvt8<BF16>(kp[v * 8], kf);
+            cvt8<BF16>(krow[swz(v * 8 + sub, t, D / 8)], kf);
 #pragma unroll
             for (int g = 0; g < GT; ++g)
 #pragma unroll
@@ -172,7 +176,7 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
             const float r = exp2f(m[g] - mx);
             l[g] *= r;
 #pragma unroll
-            for (int e = 0; e < D / 8; ++e) o[g][e] *= r;
+            for (int e = 0; e < NV * 8; ++e) o[g][e] *= r;
             m[g] = mx;
         }
     }
@@ -181,9 +185,9 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
 // o += softmax weights x V for the tile whose scores are in sc.
 template <int D, int GT, int BT, bool BF16>
 __device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp, int sub,
-                                            const float (&sc)[BT / 4][GT], float (&o)[GT][D / 8],
+                                            const float (&sc)[BT / 4][GT], float (&o)[GT][(D + 63) / 64 * 8],
                                             const float (&m)[GT], float (&l)[GT]) {
-    constexpr int NV = D / 64, NQ = BT / 4, ROW = D * 2;
+    constexpr int NV = (D + 63) / 64, NQ = BT / 4, ROW = D * 2;
 #pragma unroll
     for (int i = 0; i < NQ; ++i) {
         const int t = 4 * i + grp;
@@ -194,11 +198,12 @@ __device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp
                 pw[g] = exp2f(sc[i][g] - m[g]);
                 l[g] += pw[g];
             }
-            const uint4 *vp = reinterpret_cast<const uint4 *>(sV + t * ROW) + swz(sub, t);
+            const uint4 *vrow = reinterpret_cast<const uint4 *>(sV + t * ROW);
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
+                if ((v + 1) * 64 > D && v * 64 + sub * 8 >= D) continue;
                 float vf[8];
-                cvt8<BF16>(vp[v * 8], vf);
+                cvt8<BF16>(vrow[swz(v * 8 + sub, t, D / 8)], vf);
 #pragma unroll
                 for (int g = 0; g < GT; ++g)
 #pragma unroll
@@ -212,9 +217,10 @@ __device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp
 // Stores one row held in group layout (lanes 0..7 cover the row).
 template <int D, bool BF16>
 __device__ __forceinline__ void store_row_grouped(void *out, float *out_f32, size_t row, int sub,
-                                                  const float (&o)[D / 8], float scale) {
+                                                  const float (&o)[(D + 63) / 64 * 8], float scale) {
 #pragma unroll
-    for (int v = 0; v < D / 64; ++v) {
+    for (int v = 0; v < (D + 63) / 64; ++v) {
+        if ((v + 1) * 64 > D && v * 64 + sub * 8 >= D) continue;
         float x[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) x[e] = o[v * 8 + e] * scale;
@@ -247,7 +253,7 @@ __device__ __forceinline__ void store_row_grouped(void *out, float *out_f32, siz
 
 template <int D_, int GT_, int BT_, bool BF16_>
 struct ScalarMath {
-    static constexpr int D = D_, BT = BT_, E = D_ / 8;
+    static constexpr int D = D_, BT = BT_, NV = (D_ + 63) / 64, E = NV * 8;   // a lane owns 8 elements per 64-element span
     static constexpr bool BF16 = BF16_;
     float q[GT_][E], o[GT_][E], m[GT_], l[GT_], sc[BT_ / 4][GT_];
     int grp, sub;
@@ -265,8 +271,9 @@ struct ScalarMath {
             const uint16_t *qrow =
                 reinterpret_cast<const uint16_t *>(p.q) + ((size_t)s * p.Hq + (size_t)hg * GT_ + g) * D;
 #pragma unroll
-            for (int v = 0; v < D / 64; ++v) {
-                const uint4 r = __ldg(reinterpret_cast<const uint4 *>(qrow + v * 64 + sub * 8));
+            for (int v = 0; v < NV; ++v) {
+                const bool in = v * 64 + sub * 8 < D;
+                const uint4 r = in ? __ldg(reinterpret_cast<const uint4 *>(qrow + v * 64 + sub * 8)) : make_uint4(0, 0, 0, 0);
                 float qf[8];
                 cvt8<BF16>(r, qf);
 #pragma unroll
@@ -291,7 +298,8 @@ struct ScalarMath {
 #pragma unroll
         for (int g = 0; g < GT_; ++g) a[g] = 0.f;
 #pragma unroll
-        for (int v = 0; v < D / 64; ++v) {
+        for (int v = 0; v < NV; ++v) {
+            if (v * 64 + sub * 8 >= D) continue;
             float kf[8];
             cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(krow + v * 64 + sub * 8)), kf);
 #pragma unroll
@@ -320,7 +328,8 @@ struct ScalarMath {
                 l[g] += pw[g];
             }
 #pragma unroll
-            for (int v = 0; v < D / 64; ++v) {
+            for (int v = 0; v < NV; ++v) {
+                if (v * 64 + sub * 8 >= D) continue;
                 float vf[8];
                 cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(vrow + v * 64 + sub * 8)), vf);
 #pragma unroll
@@ -363,10 +372,12 @@ struct ScalarMath {
                 const float a1 = exp2f(m[g] - mm), a2 = exp2f(ml.x - mm);
                 l[g] = l[g] * a1 + ml.y * a2;
 #pragma unroll
-                for (int v = 0; v < D / 64; ++v)
+                for (int v = 0; v < NV; ++v) {
+                    if (v * 64 + sub * 8 >= D) continue;
 #pragma unroll
                     for (int e = 0; e < 8; ++e)
                         o[g][v * 8 + e] = o[g][v * 8 + e] * a1 + p.acc_o[row * D + v * 64 + sub * 8 + e] * a2;
+                }
                 m[g] = mm;
             }
             __syncwarp();   // all lanes have read the old state before group 0 overwrites it
@@ -502,7 +513,7 @@ struct MmaMath {
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
             uint32_t b0, b1, b2, b3;
-            ldsm_x4(rowaddr + (swz(2 * ks + half, tok) << 4), b0, b1, b2, b3);
+            ldsm_x4(rowaddr + (swz(2 * ks + half, tok, D / 8) << 4), b0, b1, b2, b3);
             mma16816<BF16>(s0, qa[ks], b0, b1);
             mma16816<BF16>(s1, qa[ks], b2, b3);
         }
@@ -554,7 +565,7 @@ struct MmaMath {
 #pragma unroll
         for (int jp = 0; jp < D / 16; ++jp) {
             uint32_t b0, b1, b2, b3;
-            ldsm_x4_t(rowaddr + (swz(2 * jp + hi, tok) << 4), b0, b1, b2, b3);
+            ldsm_x4_t(rowaddr + (swz(2 * jp + hi, tok, D / 8) << 4), b0, b1, b2, b3);
             if (ntok < BT) {   // never let unspecified bits (possibly NaN patterns) reach a product
                 b0 &= k0; b1 &= k1; b2 &= k0; b3 &= k1;
             }
@@ -686,7 +697,8 @@ struct MmaMath {
 template <int D, bool BF16>
 __device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int wf, int wf_slot, int nc, int g, int GT,
                                                    size_t row, int lane) {
-    constexpr int EPL = D / 32;
+    constexpr int EPL = D > 64 ? 4 : 2;   // lanes 0 .. D / EPL - 1 each own EPL consecutive elements
+    const bool own = lane * EPL < D;
     // contributor c is warp wf + c; the first one may have used its second slot, all others used their first
     auto slot_of = [&](int c) { return c == 0 ? 2 * wf + wf_slot : 2 * (wf + c); };
     float mm = kNegBig;
@@ -703,6 +715,7 @@ __device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int wf
         const float a = exp2f(ml.x - mm);
         ll += ml.y * a;
         const float *po = p.part_o + pr * D + lane * EPL;
+        if (!own) continue;
         if (EPL == 4) {
             const float4 x = __ldcg(reinterpret_cast<const float4 *>(po));
             acc[0] = fmaf(a, x.x, acc[0]);
@@ -716,6 +729,7 @@ __device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int wf
         }
     }
     const size_t idx = row * D + lane * EPL;
+    if (!own) return;
     if (p.finalize) {
         const float inv = ll > 0.f ? 1.f / ll : 0.f;
         if (p.out_f32) {
@@ -750,7 +764,8 @@ __device__ __forceinline__ void merge_partials_row(const DecodeParams &p, int wf
 template <int D, bool BF16, int R>
 __device__ __forceinline__ void merge_partials_rows(const DecodeParams &p, int wf, int wf_slot, int nc, int g0, int GT,
                                                     size_t row0, int lane) {
-    constexpr int EPL = D / 32;
+    constexpr int EPL = D > 64 ? 4 : 2;
+    const bool own = lane * EPL < D;
     auto slot_of = [&](int c) { return c == 0 ? 2 * wf + wf_slot : 2 * (wf + c); };
     float mm[R], ll[R], acc[R][EPL];
 #pragma unroll
@@ -778,6 +793,7 @@ __device__ __forceinline__ void merge_partials_rows(const DecodeParams &p, int w
             if (g0 + j < GT) {
                 ml[j] = __ldcg(reinterpret_cast<const float2 *>(&p.part_ml[(pr + j) * 2]));
                 const float *po = p.part_o + (pr + j) * D + lane * EPL;
+                if (!own) continue;
                 if (EPL == 4) {
                     const float4 v = __ldcg(reinterpret_cast<const float4 *>(po));
                     x[j][0] = v.x; x[j][1] = v.y; x[j][2] = v.z; x[j][3] = v.w;
@@ -800,6 +816,7 @@ __device__ __forceinline__ void merge_partials_rows(const DecodeParams &p, int w
         if (g0 + j >= GT) continue;
         const size_t row = row0 + g0 + j;
         const size_t idx = row * D + lane * EPL;
+        if (!own) continue;
         if (p.finalize) {
             const float inv = ll[j] > 0.f ? 1.f / ll[j] : 0.f;
             if (p.out_f32) {
@@ -1139,7 +1156,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
                     const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v_new : p.k_new) +
                                          ((size_t)s * p.Hkv + h) * (D * 2) + lane * 16;
                     uint8_t *dst =
-                        base + (size_t)(kv * p.Hkv + h) * TILE + (size_t)slot * (D * 2) + swz(lane, slot) * 16;
+                        base + (size_t)(kv * p.Hkv + h) * TILE + (size_t)slot * (D * 2) + swz(lane, slot, row_vecs) * 16;
                     *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
                 }
             } else if (lane == 0) {
@@ -1329,7 +1346,7 @@ __global__ void append_kernel(const AppendParams p) {
             const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
                                  ((size_t)s * p.Hkv + h) * row_bytes + vec * 16;
             uint8_t *dst =
-                base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)slot * row_bytes + swz(vec, slot) * 16;
+                base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)slot * row_bytes + swz(vec, slot, row_vecs) * 16;
             *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
         }
     } else if (threadIdx.x == 0) {
@@ -1376,7 +1393,7 @@ __global__ void fill_kernel(const FillParams p) {
         const int t = r / row_vecs, vec = r - t * row_vecs;
         const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
                              (((size_t)s * p.T + (size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
-        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + swz(vec, t) * 16;
+        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + swz(vec, t, row_vecs) * 16;
         *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
     }
 }
@@ -1396,7 +1413,7 @@ __global__ void pack_kernel(const PackParams p) {
         const int t = r / row_vecs, vec = r - t * row_vecs;
         const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v : p.k) +
                              (((size_t)s * p.T + (size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
-        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + swz(vec, t) * 16;
+        uint8_t *dst = base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + swz(vec, t, row_vecs) * 16;
         *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
     }
 }
@@ -1423,7 +1440,7 @@ __global__ void gather_kernel(const GatherParams p) {
         r -= h * ntok * row_vecs;
         const int t = r / row_vecs, vec = r - t * row_vecs;
         const uint8_t *src =
-            base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + swz(vec, t) * 16;
+            base + (size_t)(kv * p.Hkv + h) * tile_bytes + (size_t)t * row_bytes + swz(vec, t, row_vecs) * 16;
         uint8_t *dst = reinterpret_cast<uint8_t *>(kv ? p.v_out : p.k_out) +
                        (((size_t)j * p.BT + t) * p.Hkv + h) * row_bytes + vec * 16;
         *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
@@ -1455,6 +1472,7 @@ DecodeFn pick_gt(int GT, int mode) {
 DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
     if (BT != 16) return nullptr;
     if (D == 64) return bf16 ? pick_gt<64, true>(GT, mode) : pick_gt<64, false>(GT, mode);
+    if (D == 80) return bf16 ? pick_gt<80, true>(GT, mode) : pick_gt<80, false>(GT, mode);
     if (D == 128) return bf16 ? pick_gt<128, true>(GT, mode) : pick_gt<128, false>(GT, mode);
     return nullptr;
 }

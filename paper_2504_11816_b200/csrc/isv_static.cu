@@ -73,8 +73,9 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
         return err(ISV_EINVAL, "isv_attn_decode_static: pool, q and outputs must be 16-byte aligned");
     if (kv_heads < 1 || q_heads < 1 || q_heads % kv_heads != 0)
         return err(ISV_EINVAL, "isv_attn_decode_static: q_heads must be a positive multiple of kv_heads");
-    if ((head_dim != 64 && head_dim != 128) || block_tokens != 16 || (dtype != ISV_F16 && dtype != ISV_BF16))
-        return err(ISV_EINVAL, "isv_attn_decode_static: head_dim 64/128, block_tokens 16, dtype f16/bf16 only");
+    if ((head_dim != 64 && head_dim != 80 && head_dim != 128) || block_tokens != 16 ||
+        (dtype != ISV_F16 && dtype != ISV_BF16))
+        return err(ISV_EINVAL, "isv_attn_decode_static: head_dim 64/80/128, block_tokens 16, dtype f16/bf16 only");
     if (n_seqs < 0 || n_seqs > 4096 || max_blocks_per_seq < 1 || table_stride < max_blocks_per_seq ||
         n_pool_blocks < 1 || max_ctas < 0)
         return err(ISV_EINVAL, "isv_attn_decode_static: bad n_seqs (%d) or block counts (%d)", n_seqs,

@@ -63,6 +63,9 @@ CONFIGS: Dict[str, Workload] = {
     "c3": Workload("c3", 32, 32, 32, 128, "f16", 128, 2048, 2048, 64, 16, 0.5, 2, 2),
     # Llama-3-8B-shaped GQA, bf16, three quarters on the host
     "c4": Workload("c4", 32, 32, 8, 128, "bf16", 256, 4096, 4096, 32, 16, 0.75, 3, 3),
+    # the paper's own offline workload (Section V-A): OPT-2.7B (32 layers, 32 heads x 80), batch 32, 1024 input
+    # and 128 output tokens, fp16; offload fraction 0 / 0.6 / 1 in its Table VI (set with --offload)
+    "opt2.7b": Workload("opt2.7b", 32, 32, 32, 80, "f16", 32, 1024, 1024, 128, 16, 0.0, 0, 5),
     # 13B-shaped, ragged contexts, 1 % of K/V entries scaled by 8; offload fraction is swept
     "c5": Workload("c5", 40, 40, 40, 128, "f16", 64, 512, 8192, 32, 16, 0.0, 4, 4,
                    outlier_prob=0.01, outlier_scale=8.0),

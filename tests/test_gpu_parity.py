@@ -104,7 +104,7 @@ def test_result_does_not_depend_on_split_or_chunk_size(ctas, chunk_blocks):
 # 32 as two passes of 16
 @pytest.mark.parametrize("q_heads,kv_heads", [(8, 8), (8, 4), (8, 2), (16, 2), (6, 2), (32, 2), (24, 2), (10, 2),
                                               (64, 2)])
-@pytest.mark.parametrize("head_dim", [64, 128])
+@pytest.mark.parametrize("head_dim", [64, 80, 128])
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 def test_parity_over_head_grouping_head_dim_and_dtype(q_heads, kv_heads, head_dim, dtype):
     fused = (q_heads + head_dim) % 3 != 0

@@ -42,12 +42,13 @@ def _paged_pool(k_bits, v_bits, lens, kv_heads, head_dim, seed):
     stored = np.empty_like(chunks)
     for t in range(16):
         for c in range(head_dim // 8):
-            stored[:, :, :, t, c ^ (t % 8)] = chunks[:, :, :, t, c]
+            pos = c ^ (t % 8) if c < head_dim // 8 // 8 * 8 else c   # complete groups of eight chunks only
+            stored[:, :, :, t, pos] = chunks[:, :, :, t, c]
     pool = stored.reshape(total, 2, kv_heads, 16, head_dim)
     return pool, table, total, stride, max(nb)
 
 
-@pytest.mark.parametrize("q_heads,kv_heads,head_dim,dtype", [(8, 8, 128, "f16"), (8, 2, 64, "bf16")])
+@pytest.mark.parametrize("q_heads,kv_heads,head_dim,dtype", [(8, 8, 128, "f16"), (8, 2, 64, "bf16"), (4, 4, 80, "f16")])
 def test_static_entry_matches_handle_entry_on_two_calls_in_a_row(q_heads, kv_heads, head_dim, dtype):
     lens = [300, 1, 16, 513, 77]
     w = W.Workload("na", 1, q_heads, kv_heads, head_dim, dtype, len(lens), 1, 513, 2, 16, 0.0, 0, 31)
