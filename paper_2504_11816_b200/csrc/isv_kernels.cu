@@ -130,8 +130,13 @@ __device__ __forceinline__ int swz(int chunk, int t, int nchunks) {
 // ---------------------------------------------------------------- one K tile, one V tile
 
 // Lane layout inside a warp: grp = lane / 8 owns tokens grp, grp+4, ... of the
-// tile; sub = lane % 8 owns head-dim elements [v*64 + sub*8, +8) for v < D/64.
-// Each group keeps its own running (m, l, o); groups are merged at unit end.
+// tile; sub = lane % 8 owns head-dim elements [v*64 + sub*8, +8) of every complete
+// 64-element span v.  Each group keeps its own running (m, l, o); groups are merged at unit end.
+// head_dim 80 leaves a tail of 16 elements = 2 chunks per token.  Giving it to lanes sub 0 and 1 of every
+// pass would cost a whole span's instructions for a quarter of the lanes, so the tails of a group's four
+// tokens are handled in one extra step instead: lane sub takes the tail chunk (sub & 1) of the token of
+// pass sub / 2.  Its registers q[.][NVF*8 ..] / o[.][NVF*8 ..] then belong to elements
+// NVF*64 + (sub & 1)*8 .., and the o tails of the lanes with equal sub & 1 are summed at unit end.
 
 // Scores of the tile's tokens against the GT query heads (log2 domain, q is
 // pre-scaled), and the running maximum brought up to date (o and l rescaled).
@@ -139,7 +144,8 @@ template <int D, int GT, int BT, bool BF16>
 __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp, int sub,
                                             const float (&q)[GT][(D + 63) / 64 * 8], float (&sc)[BT / 4][GT],
                                             float (&o)[GT][(D + 63) / 64 * 8], float (&m)[GT], float (&l)[GT]) {
-    constexpr int NV = (D + 63) / 64, NQ = BT / 4, ROW = D * 2;
+    constexpr int NVF = D / 64, NV = (D + 63) / 64, NQ = BT / 4, ROW = D * 2;
+    static_assert(D % 64 == 0 || D % 64 == 16, "head_dim: whole 64-element spans, plus at most a 16-element tail");
 #pragma unroll
     for (int i = 0; i < NQ; ++i) {
         const int t = 4 * i + grp;
@@ -148,8 +154,7 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
 #pragma unroll
         for (int g = 0; g < GT; ++g) a0[g] = a1[g] = 0.f;
 #pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            if ((v + 1) * 64 > D && v * 64 + sub * 8 >= D) continue;   // last, incomplete 64-element span
+        for (int v = 0; v < NVF; ++v) {
             float kf[8];
             cvt8<BF16>(krow[swz(v * 8 + sub, t, D / 8)], kf);
 #pragma unroll
@@ -164,9 +169,29 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
             a += __shfl_xor_sync(kFull, a, 4);
             a += __shfl_xor_sync(kFull, a, 2);
             a += __shfl_xor_sync(kFull, a, 1);
-            sc[i][g] = (t < ntok) ? a : kNegBig;
+            sc[i][g] = a;
         }
     }
+    if (NV > NVF) {   // the 16-element tails of the group's four tokens, one chunk per lane
+        const int tt = 4 * (sub >> 1) + grp;
+        float kf[8];
+        cvt8<BF16>(reinterpret_cast<const uint4 *>(sK + tt * ROW)[NVF * 8 + (sub & 1)], kf);
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            float tp = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) tp = fmaf(q[g][NVF * 8 + e], kf[e], tp);
+            tp += __shfl_xor_sync(kFull, tp, 1);   // lanes 2i and 2i+1 of the group: tail of the token of pass i
+#pragma unroll
+            for (int i = 0; i < NQ; ++i) sc[i][g] += __shfl_sync(kFull, tp, grp * 8 + 2 * i);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < NQ; ++i)   // slots past the sequence end hold unspecified bits: their scores are replaced
+        if (4 * i + grp >= ntok) {
+#pragma unroll
+            for (int g = 0; g < GT; ++g) sc[i][g] = kNegBig;
+        }
 #pragma unroll
     for (int g = 0; g < GT; ++g) {
         float mx = sc[0][g];
@@ -187,28 +212,43 @@ template <int D, int GT, int BT, bool BF16>
 __device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp, int sub,
                                             const float (&sc)[BT / 4][GT], float (&o)[GT][(D + 63) / 64 * 8],
                                             const float (&m)[GT], float (&l)[GT]) {
-    constexpr int NV = (D + 63) / 64, NQ = BT / 4, ROW = D * 2;
+    constexpr int NVF = D / 64, NV = (D + 63) / 64, NQ = BT / 4, ROW = D * 2;
+    float pwv[NQ][GT];   // the weights of the four passes (used again by the tail step)
 #pragma unroll
     for (int i = 0; i < NQ; ++i) {
         const int t = 4 * i + grp;
+#pragma unroll
+        for (int g = 0; g < GT; ++g) pwv[i][g] = 0.f;
         if (t < ntok) {   // slots past the sequence end hold unspecified bits: never touch them
-            float pw[GT];
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
-                pw[g] = exp2f(sc[i][g] - m[g]);
-                l[g] += pw[g];
+                pwv[i][g] = exp2f(sc[i][g] - m[g]);
+                l[g] += pwv[i][g];
             }
             const uint4 *vrow = reinterpret_cast<const uint4 *>(sV + t * ROW);
 #pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                if ((v + 1) * 64 > D && v * 64 + sub * 8 >= D) continue;
+            for (int v = 0; v < NVF; ++v) {
                 float vf[8];
                 cvt8<BF16>(vrow[swz(v * 8 + sub, t, D / 8)], vf);
 #pragma unroll
                 for (int g = 0; g < GT; ++g)
 #pragma unroll
                     for (int e = 0; e < 8; e += 2)
-                        ffma2(o[g][v * 8 + e], o[g][v * 8 + e + 1], pw[g], pw[g], vf[e], vf[e + 1]);
+                        ffma2(o[g][v * 8 + e], o[g][v * 8 + e + 1], pwv[i][g], pwv[i][g], vf[e], vf[e + 1]);
+            }
+        }
+    }
+    if (NV > NVF) {
+        const int pi = sub >> 1, tt = 4 * pi + grp;
+        if (tt < ntok) {
+            float vf[8];
+            cvt8<BF16>(reinterpret_cast<const uint4 *>(sV + tt * ROW)[NVF * 8 + (sub & 1)], vf);
+#pragma unroll
+            for (int g = 0; g < GT; ++g) {
+                const float pw = pi == 0 ? pwv[0][g] : pi == 1 ? pwv[1][g] : pi == 2 ? pwv[2][g] : pwv[3][g];
+#pragma unroll
+                for (int e = 0; e < 8; e += 2)
+                    ffma2(o[g][NVF * 8 + e], o[g][NVF * 8 + e + 1], pw, pw, vf[e], vf[e + 1]);
             }
         }
     }
@@ -253,7 +293,7 @@ __device__ __forceinline__ void store_row_grouped(void *out, float *out_f32, siz
 
 template <int D_, int GT_, int BT_, bool BF16_>
 struct ScalarMath {
-    static constexpr int D = D_, BT = BT_, NV = (D_ + 63) / 64, E = NV * 8;   // a lane owns 8 elements per 64-element span
+    static constexpr int D = D_, BT = BT_, NVF = D_ / 64, NV = (D_ + 63) / 64, E = NV * 8;   // 8 elements per span and lane
     static constexpr bool BF16 = BF16_;
     float q[GT_][E], o[GT_][E], m[GT_], l[GT_], sc[BT_ / 4][GT_];
     int grp, sub;
@@ -272,8 +312,8 @@ struct ScalarMath {
                 reinterpret_cast<const uint16_t *>(p.q) + ((size_t)s * p.Hq + (size_t)hg * GT_ + g) * D;
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
-                const bool in = v * 64 + sub * 8 < D;
-                const uint4 r = in ? __ldg(reinterpret_cast<const uint4 *>(qrow + v * 64 + sub * 8)) : make_uint4(0, 0, 0, 0);
+                // complete spans: elements v*64 + sub*8 ..; the tail span: chunk sub & 1 in every lane
+                const uint4 r = __ldg(reinterpret_cast<const uint4 *>(qrow + v * 64 + (v < NVF ? sub : (sub & 1)) * 8));
                 float qf[8];
                 cvt8<BF16>(r, qf);
 #pragma unroll
@@ -299,7 +339,7 @@ struct ScalarMath {
         for (int g = 0; g < GT_; ++g) a[g] = 0.f;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
-            if (v * 64 + sub * 8 >= D) continue;
+            if (v * 64 + sub * 8 >= D) continue;   // the tail is counted once: by lanes sub 0 and 1
             float kf[8];
             cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(krow + v * 64 + sub * 8)), kf);
 #pragma unroll
@@ -341,6 +381,17 @@ struct ScalarMath {
     }
     // End of a unit: merge the four token groups of the warp (every group ends with the merged state).
     __device__ __forceinline__ void finish() {
+        if (NV > NVF) {   // tail elements: sum the shares of the lanes with equal sub & 1
+#pragma unroll
+            for (int g = 0; g < GT_; ++g)
+#pragma unroll
+                for (int e = NVF * 8; e < E; ++e) {
+                    float x = o[g][e];
+                    x += __shfl_xor_sync(kFull, x, 2);
+                    x += __shfl_xor_sync(kFull, x, 4);
+                    o[g][e] = x;
+                }
+        }
 #pragma unroll
         for (int g = 0; g < GT_; ++g) {
             float mm = fmaxf(m[g], __shfl_xor_sync(kFull, m[g], 8));
