@@ -933,11 +933,21 @@ int isv_decode_step_host(isv_kv *h, const void *q, const void *k, const void *v,
         if ((rc = dev_alloc((void **)&h->step_buf, 2 * qs_max + 2 * ks_max, &h->scratch_bytes, "step buffers"))) return rc;
     }
     uint8_t *dq = h->step_buf, *dout = dq + qs_max, *dk = dout + qs_max, *dv = dk + ks_max;
-    // Inputs travel in groups of a few layers on their own stream and results go back on the
-    // write-back stream, so that only the first group's copy and the last group's read-back are
-    // not hidden behind the attention of the other layers.
-    const int group = 4;
-    const int n_groups = (g.layers + group - 1) / group;
+    // Inputs travel in groups of layers on their own stream and results go back on the write-back stream,
+    // so that only the first group's copy and the last group's read-back are not hidden behind the attention
+    // of the other layers.  Those two groups are a single layer; in between the groups grow to eight layers
+    // (every group boundary is a cross-stream wait, which costs the launch overlap between two layers).
+    std::vector<int> first;   // first layer of each group, and the end
+    {
+        int l = 0;
+        const int head[2] = {1, 3};
+        for (int i = 0; i < 2 && l < g.layers; ++i) { first.push_back(l); l += std::min(head[i], g.layers - l); }
+        while (g.layers - l > 9) { first.push_back(l); l += 8; }
+        if (g.layers - l > 1) { first.push_back(l); l = g.layers - 1; }
+        if (l < g.layers) { first.push_back(l); l = g.layers; }
+        first.push_back(g.layers);
+    }
+    const int n_groups = (int)first.size() - 1;
     if (h->ev_step_in.empty()) {
         h->ev_step_in.resize(n_groups);
         h->ev_step_out.resize(n_groups);
@@ -953,14 +963,14 @@ int isv_decode_step_host(isv_kv *h, const void *q, const void *k, const void *v,
     CU(cudaEventRecord(h->ev_app, h->s_compute));
     CU(cudaStreamWaitEvent(h->s_in, h->ev_app, 0));
     for (int gi = 0; gi < n_groups; ++gi) {
-        const int l0 = gi * group, nl = std::min(group, g.layers - l0);
+        const int l0 = first[gi], nl = first[gi + 1] - l0;
         CU(cudaMemcpyAsync(dk + l0 * kl, (const uint8_t *)k + l0 * kl, nl * kl, cudaMemcpyHostToDevice, h->s_in));
         CU(cudaMemcpyAsync(dv + l0 * kl, (const uint8_t *)v + l0 * kl, nl * kl, cudaMemcpyHostToDevice, h->s_in));
         CU(cudaMemcpyAsync(dq + l0 * ql, (const uint8_t *)q + l0 * ql, nl * ql, cudaMemcpyHostToDevice, h->s_in));
         CU(cudaEventRecord(h->ev_step_in[gi], h->s_in));
     }
     for (int gi = 0; gi < n_groups; ++gi) {
-        const int l0 = gi * group, nl = std::min(group, g.layers - l0);
+        const int l0 = first[gi], nl = first[gi + 1] - l0;
         CU(cudaStreamWaitEvent(h->s_compute, h->ev_step_in[gi], 0));
         for (int l = l0; l < l0 + nl; ++l)
             if ((rc = isv_decode_layer(h, l, dq + l * ql, dk + l * kl, dv + l * kl, dout + l * ql, nullptr, n_seqs)))
