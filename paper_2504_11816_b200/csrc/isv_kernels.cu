@@ -1517,7 +1517,7 @@ DecodeFn pick_mode(int mode) {
 template <int D, bool BF16>
 DecodeFn pick_gt(int GT, int mode) {
     if (GT == 1) return pick_mode<ScalarMath<D, 1, 16, BF16>, ISV_WARPS_GT1>(mode);
-    if (GT >= 2 && GT <= 16) return pick_mode<MmaMath<D, BF16>, (D == 64 ? 16 : ISV_WARPS_MMA)>(mode);
+    if (GT >= 2 && GT <= 16) return pick_mode<MmaMath<D, BF16>, (D == 64 ? 16 : D == 80 ? 12 : ISV_WARPS_MMA)>(mode);
     return nullptr;
 }
 DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
@@ -1532,7 +1532,7 @@ DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
 
 // The tensor-core variant keeps 96 accumulator and operand registers per thread at head_dim 128 (8 warps);
 // at head_dim 64 it fits 128 registers, and 16 warps hide its per-visit latencies.
-int decode_warps(int GT, int D) { return GT == 1 ? ISV_WARPS_GT1 : (D == 64 ? 16 : ISV_WARPS_MMA); }
+int decode_warps(int GT, int D) { return GT == 1 ? ISV_WARPS_GT1 : (D == 64 ? 16 : D == 80 ? 12 : ISV_WARPS_MMA); }
 
 int decode_default_stages(int D, int BT, int GT) {
     const int per_stage = decode_warps(GT, D) * BT * D * 2;
