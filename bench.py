@@ -421,8 +421,8 @@ def run_ours(args, w):
     # -------- CPU reference beside it (rank 0, single-GPU runs only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        # C2: the whole batch, i.e. one full layer-step; the larger shapes: 4 sequences scaled up
-        n_sample = w.batch if w.name in ("c2", "tiny") else min(w.batch, 4)
+        # C2 and the OPT-2.7B shape: the whole batch, i.e. one full layer-step; the larger shapes: 4 sequences scaled up
+        n_sample = w.batch if w.name in ("c2", "tiny", "opt2.7b") else min(w.batch, 4)
         tps, t, threads, what = time_reference(w, n_sample, 3, 1)
         tps1, t1_, _, what1 = time_reference(w, min(w.batch, 2), 1, 0, n_threads=1)
         cpu = {"value": tps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what,

@@ -169,3 +169,13 @@ def test_pool_sizes_follow_the_kv_size_formula():
         assert info.host_blocks == info.hbm_blocks == 8 * 5
     finally:
         B.isv_kv_free(h)
+    # the paper's main model, OPT-2.7B (h1 = 2560 = 32 heads x 80, 32 layers), at its offline workload:
+    # batch 32, 1024 + 128 tokens, everything resident
+    h = _alloc(layers=32, offload_frac=0.0, max_seqs=32, max_tokens_per_seq=1152, q_heads=32, kv_heads=32,
+               head_dim=80)
+    try:
+        info = B.isv_kv_info(h)
+        assert info.kv_bytes_per_token == 2 * 2560 * 2 and info.block_bytes == 16 * 2 * 2560 * 2
+        assert info.hbm_pool_bytes == pm.kv_cache_bytes(32, 1152, 2560, 2, 32)
+    finally:
+        B.isv_kv_free(h)
