@@ -101,6 +101,9 @@ def main():
     ap.add_argument("--out-len", type=int, default=128)
     ap.add_argument("--offload", type=float, default=0.5)
     ap.add_argument("--layers", type=int, default=8)
+    ap.add_argument("--head-dim", type=int, default=128, choices=[64, 80, 128],
+                    help="32 heads of this size: 128 gives h1 = 4096; 80 gives h1 = 2560, h2 = 10240, the OPT-2.7B "
+                         "shape the paper validates its calibration on (subsection 'CTCF Validation')")
     ap.add_argument("--flops", type=float, default=2.25e15, help="FLOP/s the model divides by (dense fp16 peak)")
     args = ap.parse_args()
     import torch
@@ -110,7 +113,7 @@ def main():
     assert torch.cuda.is_available(), "calibration needs a CUDA device"
     h2d, d2h = B.isv_link_probe(1 << 30, 10)
     hw = cm.Machine(flops=args.flops, bw_h2d=h2d * 1e9, bw_d2h=d2h * 1e9)
-    base = W.Workload("cal", args.layers, 32, 32, 128, "f16", 1, args.ctx, args.ctx, args.out_len, 16, 0.0, 0, 7)
+    base = W.Workload("cal", args.layers, 32, 32, args.head_dim, "f16", 1, args.ctx, args.ctx, args.out_len, 16, 0.0, 0, 7)
     shape = cm.ModelShape(h1=base.kv_heads * base.head_dim, h2=4 * base.kv_heads * base.head_dim,
                           n_layers=base.layers, prec_bytes=2)
     steps, warmup = 8, 3
