@@ -100,7 +100,7 @@ def test_result_does_not_depend_on_split_or_chunk_size(ctas, chunk_blocks):
 
 # ---------------------------------------------------------------- head grouping, head dim, dtype
 
-# query heads per KV head: 1 and 2 run on the CUDA cores, 3..16 as one tensor-core tile (4, 8, 3, 16, 12, 5),
+# query heads per KV head: 1 runs on the CUDA cores, 2..16 as one tensor-core tile (2, 4, 8, 3, 16, 12, 5),
 # 32 as two passes of 16
 @pytest.mark.parametrize("q_heads,kv_heads", [(8, 8), (8, 4), (8, 2), (16, 2), (6, 2), (32, 2), (24, 2), (10, 2),
                                               (64, 2)])
@@ -154,12 +154,15 @@ def test_identical_query_heads_of_a_group_give_identical_outputs():
 # ---------------------------------------------------------------- special cases of the method
 
 @pytest.mark.parametrize("f", [0.0, 1.0])
-@pytest.mark.parametrize("q_heads", [4, 8])
-def test_context_of_one_token_returns_v_exactly(f, q_heads):
-    w = small(batch=3, steps=1, f=f, layers=1, q_heads=q_heads, kv_heads=2, head_dim=64, ctx=(0, 0))
+@pytest.mark.parametrize("q_heads,head_dim", [(2, 64), (4, 64), (8, 64), (2, 80), (8, 128)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_context_of_one_token_returns_v_exactly(f, q_heads, head_dim, fused):
+    # 1, 2 and 4 query heads per KV head (CUDA-core and tensor-core arithmetic); fused: the token is attended to
+    # from the caller's rows, in a visit that carries no tile
+    w = small(batch=3, steps=1, f=f, layers=1, q_heads=q_heads, kv_heads=2, head_dim=head_dim, ctx=(0, 0))
     with Harness(w, lens=[0, 0, 0]) as hz:
         hz.fill()
-        res = hz.step()                                   # the appended token is the whole context
+        res = hz.step(fused=fused)                        # the appended token is the whole context
         q, of, o16, _ = res[0]
         kb, vb = zip(*[hz.shadow.gathered(0, s) for s in range(w.batch)])
         for s in range(w.batch):
