@@ -37,14 +37,14 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the resident decode kernel from one ncu capture (bytes per KV byte
 # processed), valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernels_sha1": "3348ca26db3b9db36b5c9dccf49f39b9867b4122",
-               # multi-head shapes (CUDA-core arithmetic): (546.93 MB read + 4.68 MB written) / 539.23 MB
+NCU_TRAFFIC = {"kernels_sha1": "315a5d0284e8aa65b79e1e1cba0d9bbe00020e71",
+               # multi-head shapes (CUDA-core arithmetic): (546.94 MB read + 4.85 MB written) / 539.23 MB
                # algorithmic, 2-layer case of the default shape
-               "dram_bytes_per_kv_byte": (546.932736 + 4.678912) / 539.230208,
+               "dram_bytes_per_kv_byte": (546.935296 + 4.850688) / 539.230208,
                "source": "profiles/decode_kernel_c2_2layers.md",
-               # grouped-query shapes (tensor-core arithmetic): (540.02 MB + 4.79 MB) / 537.46 MB, 32 sequences
+               # grouped-query shapes (tensor-core arithmetic): (540.00 MB + 5.09 MB) / 537.46 MB, 32 sequences
                # and 2 layers of the 8B-GQA shape
-               "dram_bytes_per_kv_byte_gqa": (540.023296 + 4.787968) / 537.460736,
+               "dram_bytes_per_kv_byte_gqa": (539.998464 + 5.091072) / 537.460736,
                "source_gqa": "profiles/decode_kernel_gqa_c4shape_batch32_2layers.md"}
 
 

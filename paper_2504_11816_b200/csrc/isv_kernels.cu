@@ -1530,8 +1530,9 @@ DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
 
 }  // namespace
 
-// The tensor-core variant keeps 96 accumulator and operand registers per thread at head_dim 128 (8 warps);
-// at head_dim 64 it fits 128 registers, and 16 warps hide its per-visit latencies.
+// The tensor-core variant keeps 96 accumulator and operand registers per thread at head_dim 128 (8 warps),
+// 60 at head_dim 80 (12 warps fit without spills); at head_dim 64 it fits 128 registers, and 16 warps hide
+// its per-visit latencies (a visit carries only 4 KiB there).
 int decode_warps(int GT, int D) { return GT == 1 ? ISV_WARPS_GT1 : (D == 64 ? 16 : D == 80 ? 12 : ISV_WARPS_MMA); }
 
 int decode_default_stages(int D, int BT, int GT) {
