@@ -79,10 +79,11 @@ def test_reading_host_blocks_in_place_gives_the_same_result(f):
 
 @pytest.mark.parametrize("ctas", [1, 2, 7, 0])
 @pytest.mark.parametrize("chunk_blocks", [1, 0])
-def test_result_does_not_depend_on_split_or_chunk_size(ctas, chunk_blocks):
+@pytest.mark.parametrize("q_heads", [8, 32])
+def test_result_does_not_depend_on_split_or_chunk_size(ctas, chunk_blocks, q_heads):
     lens = [700, 33, 512, 129]
     outs = []
-    w = small(batch=4, steps=2, f=0.5, perm=3, ctx=(1, 700), layers=1, q_heads=8, kv_heads=8, head_dim=64)
+    w = small(batch=4, steps=2, f=0.5, perm=3, ctx=(1, 700), layers=1, q_heads=q_heads, kv_heads=8, head_dim=64)
     block_bytes = 2 * w.kv_heads * 16 * w.head_dim * 2
     with Harness(w, lens=lens, max_ctas=ctas, chunk_bytes=chunk_blocks * block_bytes) as hz:
         hz.fill()
