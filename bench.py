@@ -294,7 +294,7 @@ def run_ours(args, w):
     # -------- pass 1: device-resident inputs, no per-layer events -> `value`
     fill(measure_store=w.offload_frac > 0)
     for i in range(Wm):
-        B.isv_decode_step(h, qs[i % n_in], ks[i % n_in], vs[i % n_in], out, w.batch)
+        B.isv_decode_step(h, qs[i % n_in], ks[i % n_in], vs[i % n_in], out, None, w.batch)
     B.isv_sync(h)
     probe_before = B.isv_link_probe(1 << 30, 10) if w.offload_frac > 0 else None
     h2d_before = probe_before[0] if probe_before else None
@@ -306,7 +306,7 @@ def run_ours(args, w):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for i in range(K):
-        B.isv_decode_step(h, qs[i % n_in], ks[i % n_in], vs[i % n_in], out, w.batch)
+        B.isv_decode_step(h, qs[i % n_in], ks[i % n_in], vs[i % n_in], out, None, w.batch)
     e1.record(stream)
     barrier()
     clocks = sampler.stop()
@@ -321,12 +321,12 @@ def run_ours(args, w):
     fill()
     B.isv_set_timing(h, True)
     for i in range(Wm):
-        B.isv_decode_step(h, qs[i % n_in], ks[i % n_in], vs[i % n_in], out, w.batch)
+        B.isv_decode_step(h, qs[i % n_in], ks[i % n_in], vs[i % n_in], out, None, w.batch)
     B.isv_sync(h)
     t_res = t_h2d = t_off = t_merge = t_app = t_tot = 0.0
     staged = 0
     for i in range(K):
-        B.isv_decode_step(h, qs[i % n_in], ks[i % n_in], vs[i % n_in], out, w.batch)
+        B.isv_decode_step(h, qs[i % n_in], ks[i % n_in], vs[i % n_in], out, None, w.batch)
         st = B.isv_step_timing(h, -1)
         t_res += st.attn_resident_ms
         t_h2d += st.h2d_ms

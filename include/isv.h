@@ -49,10 +49,11 @@ extern "C" {
 #define ISV_OK               0
 #define ISV_EINVAL          (-1)   /* bad argument                                   */
 #define ISV_ENOMEM_DEVICE   (-2)   /* cudaMalloc refused                             */
-#define ISV_ENOMEM_PINNED   (-3)   /* pinned host allocation refused                 */
+#define ISV_ENOMEM_PINNED   (-3)   /* pinned host allocation refused (by the system, or because it  */
+                                   /* exceeds the environment variable ISV_PINNED_LIMIT_BYTES)      */
 #define ISV_ECAPACITY       (-4)   /* sequence or pool would exceed its capacity     */
 #define ISV_ECUDA           (-5)   /* a CUDA runtime call failed                     */
-#define ISV_ETIMEOUT        (-6)   /* a bounded wait ran out                         */
+#define ISV_ETIMEOUT        (-6)   /* a host-side wait exceeded isv_set_host_timeout */
 #define ISV_EDEVICE_STATUS  (-7)   /* a kernel reported a problem (see status bits)  */
 #define ISV_ENODEVICE       (-8)   /* compute requested on a plan-only handle        */
 
@@ -65,6 +66,8 @@ extern "C" {
 /* bits of the device status word (isv_step_times.status, isv_sync, isv_linear_status) */
 #define ISV_STATUS_BAD_BLOCK_ID  1u   /* a table entry pointed outside its pool; block skipped */
 #define ISV_STATUS_WAIT_EXPIRED  2u   /* a bounded wait inside a kernel gave up                */
+#define ISV_STATUS_BAD_LENGTH    4u   /* a device-side sequence length was negative or exceeded */
+                                      /* the table row; it was clamped to what the row covers  */
 
 typedef struct isv_kv isv_kv;   /* opaque; created by isv_kv_alloc, destroyed by isv_kv_free */
 
@@ -230,16 +233,19 @@ int isv_decode_layer(isv_kv *h, int32_t layer, const void *q_dev, const void *k_
 int isv_set_zero_copy(isv_kv *h, int32_t on);
 
 /* One decode step of all layers: isv_decode_layer for l in 0..layers-1.
- * Device arrays: q, out [layers][n_seqs][q_heads][head_dim];
- * k, v [layers][n_seqs][kv_heads][head_dim]. */
+ * Device arrays: q, out (16-bit) and out_f32 (fp32) [layers][n_seqs][q_heads][head_dim];
+ * k, v [layers][n_seqs][kv_heads][head_dim].  out_dev and out_f32_dev may each be NULL, not both. */
 int isv_decode_step(isv_kv *h, const void *q_dev, const void *k_dev, const void *v_dev,
-                    void *out_dev, int32_t n_seqs);
+                    void *out_dev, float *out_f32_dev, int32_t n_seqs);
 
 /* The same step with HOST buffers of the same shapes (pinned memory gives
  * asynchronous copies): inputs are copied to library-owned device buffers a
  * few layers at a time on a copy stream while earlier layers compute, and
  * each group's result is copied back as soon as it is ready.  Returns after
- * the whole result is in out_host (synchronises). */
+ * the whole result is in out_host (synchronises).  The first call on a handle
+ * allocates the device buffers for one step's q, k, v and out (cudaMalloc,
+ * counted in isv_kv_info's scratch_bytes) and a copy stream; make it outside
+ * any region that must not allocate. */
 int isv_decode_step_host(isv_kv *h, const void *q_host, const void *k_host,
                          const void *v_host, void *out_host, int32_t n_seqs);
 
@@ -280,6 +286,27 @@ int isv_step_timing(isv_kv *h, int32_t layer, isv_step_times *out);
 /* Waits for everything enqueued by the handle; returns ISV_EDEVICE_STATUS if
  * a kernel flagged a problem since the last call (bits in *status_out). */
 int isv_sync(isv_kv *h, uint32_t *status_out);
+
+/* ---- failure handling ----------------------------------------------------- */
+
+/* Limit, in seconds, of every host-side wait of this handle (isv_sync, isv_step_timing, isv_kv_fill,
+ * isv_fill_timing, isv_kv_gather, isv_decode_step_host): a wait that exceeds it returns ISV_ETIMEOUT
+ * and leaves the work enqueued, so the caller can wait again, report, or tear down.  0 (the default)
+ * waits without limit.  The wait polls the stream instead of blocking in the driver. */
+int isv_set_host_timeout(isv_kv *h, double seconds);
+
+/* Limit of a device-side wait for a K/V copy, in polls of its barrier (0 = the built-in default, about
+ * 4 million polls, i.e. seconds).  A warp whose wait runs out sets ISV_STATUS_WAIT_EXPIRED, gives its
+ * other copies one more bounded chance to land and leaves the kernel; the handle stays usable and the
+ * next isv_sync / isv_step_timing returns ISV_EDEVICE_STATUS once and clears the state.  The outputs of
+ * that launch are incomplete. */
+int isv_set_wait_limit(isv_kv *h, uint32_t polls);
+
+/* Failure injection for tests of the path above: in each of the next `launches` resident attention
+ * launches one warp arms the barrier of its first K tile without issuing the copy, as if the transfer
+ * had been lost; its wait then runs out after the limit set by isv_set_wait_limit.  Nothing faults
+ * and nothing hangs. */
+int isv_inject_lost_copy(isv_kv *h, int32_t launches);
 
 /* Measures pinned host<->device copy bandwidth on the current device: `bytes`
  * per copy, best of `reps`, CUDA events.  This is the measured host-link rate

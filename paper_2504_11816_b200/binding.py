@@ -30,6 +30,9 @@ ISV_F16 = 0
 ISV_BF16 = 1
 ISV_BLOCK_NONE = -1
 ISV_BLOCK_HOST_BIT = 1 << 30
+ISV_STATUS_BAD_BLOCK_ID = 1
+ISV_STATUS_WAIT_EXPIRED = 2
+ISV_STATUS_BAD_LENGTH = 4
 
 EXPORTS = [
     "isv_kv_alloc", "isv_kv_free", "isv_kv_reset", "isv_kv_info", "isv_kv_fill", "isv_kv_fill_async",
@@ -37,6 +40,7 @@ EXPORTS = [
     "isv_attn_decode", "isv_decode_layer", "isv_decode_step", "isv_decode_step_host", "isv_kv_gather",
     "isv_block_table_dev", "isv_seq_lens_dev", "isv_block_table_host", "isv_seq_lens_host",
     "isv_plan_bytes", "isv_set_zero_copy", "isv_set_timing", "isv_step_timing", "isv_sync", "isv_link_probe",
+    "isv_set_host_timeout", "isv_set_wait_limit", "isv_inject_lost_copy",
     "isv_attn_decode_static", "isv_linear_create", "isv_linear_forward", "isv_linear_status", "isv_linear_free",
     "isv_last_error",
 ]
@@ -121,7 +125,7 @@ def lib():
     L.isv_kv_append.argtypes = [vp, i32, vp, vp, i32]
     L.isv_attn_decode.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32]
     L.isv_decode_layer.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32]
-    L.isv_decode_step.argtypes = [vp, vp, vp, vp, vp, i32]
+    L.isv_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, i32]
     L.isv_decode_step_host.argtypes = [vp, vp, vp, vp, vp, i32]
     L.isv_kv_gather.argtypes = [vp, i32, i32, vp, vp, P(i32)]
     L.isv_block_table_dev.argtypes = [vp, P(i32)]
@@ -133,6 +137,9 @@ def lib():
     L.isv_plan_bytes.argtypes = [vp, i32, i32, P(u64), P(u64), P(u64), P(i32)]
     L.isv_set_zero_copy.argtypes = [vp, i32]
     L.isv_set_timing.argtypes = [vp, i32]
+    L.isv_set_host_timeout.argtypes = [vp, ctypes.c_double]
+    L.isv_set_wait_limit.argtypes = [vp, ctypes.c_uint32]
+    L.isv_inject_lost_copy.argtypes = [vp, i32]
     L.isv_step_timing.argtypes = [vp, i32, P(StepTimes)]
     L.isv_sync.argtypes = [vp, P(ctypes.c_uint32)]
     L.isv_link_probe.argtypes = [u64, i32, P(ctypes.c_double), P(ctypes.c_double)]
@@ -230,8 +237,8 @@ def isv_decode_layer(h: int, layer: int, q, k, v, out, out_f32, n_seqs: int):
     _check(lib().isv_decode_layer(h, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(out_f32), n_seqs))
 
 
-def isv_decode_step(h: int, q, k, v, out, n_seqs: int):
-    _check(lib().isv_decode_step(h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), n_seqs))
+def isv_decode_step(h: int, q, k, v, out, out_f32, n_seqs: int):
+    _check(lib().isv_decode_step(h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(out_f32), n_seqs))
 
 
 def isv_decode_step_host(h: int, q, k, v, out, n_seqs: int):
@@ -278,6 +285,18 @@ def isv_plan_bytes(h: int, layer: int, n_seqs: int):
 
 def isv_set_zero_copy(h: int, on: bool):
     _check(lib().isv_set_zero_copy(h, 1 if on else 0))
+
+
+def isv_set_host_timeout(h: int, seconds: float):
+    _check(lib().isv_set_host_timeout(h, float(seconds)))
+
+
+def isv_set_wait_limit(h: int, polls: int):
+    _check(lib().isv_set_wait_limit(h, polls))
+
+
+def isv_inject_lost_copy(h: int, launches: int):
+    _check(lib().isv_inject_lost_copy(h, launches))
 
 
 def isv_set_timing(h: int, on: bool):

@@ -43,11 +43,11 @@ def measure(w, steps: int, warmup: int):
         torch.cuda.synchronize()
         B.isv_set_timing(h, True)
         for _ in range(warmup):
-            B.isv_decode_step(h, q, k, v, out, w.batch)
+            B.isv_decode_step(h, q, k, v, out, None, w.batch)
         B.isv_sync(h)
         acc = {"attn": 0.0, "h2d": 0.0, "total": 0.0, "bytes_res": 0, "bytes_off": 0}
         for _ in range(steps):
-            B.isv_decode_step(h, q, k, v, out, w.batch)
+            B.isv_decode_step(h, q, k, v, out, None, w.batch)
             st = B.isv_step_timing(h, -1)
             acc["attn"] += (st.attn_resident_ms + st.merge_ms) * 1e-3
             acc["h2d"] += st.h2d_ms * 1e-3

@@ -3,6 +3,7 @@
 // isv_kernels.cu; there is no CPU path for attention.
 #include <cuda_runtime.h>
 
+#include <chrono>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -10,6 +11,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <thread>
 #include <vector>
 
 #include "../../include/isv.h"
@@ -105,6 +107,10 @@ struct isv_kv {
     uint64_t launches = 0;                 // kernels launched so far
     int last_fused_layer = -1;             // layer of the latest fused decode launch if nothing else of ours
                                            // was launched on the compute stream since, else -1
+    // failure handling
+    double host_timeout_s = 0.0;           // limit of a host-side wait; 0 = none
+    uint32_t spin_limit = 0;               // device-side wait limit in polls; 0 = the kernels' default
+    int lost_copies = 0;                   // failure injection: resident launches still to lose a copy
     // timing
     bool timing = false;
     std::vector<LayerEvents> lev;
@@ -197,6 +203,20 @@ int pick_stages(const Geometry &g, int mode, int smem_limit, size_t *smem_out) {
     return best;
 }
 
+// ISV_PINNED_LIMIT_BYTES caps the host KV pool the way a locked-memory limit of the system would: a
+// pool beyond it is refused before anything is allocated.
+int check_pinned_limit(uint64_t bytes) {
+    const char *e = getenv("ISV_PINNED_LIMIT_BYTES");
+    if (!e || !*e) return ISV_OK;
+    const unsigned long long lim = strtoull(e, nullptr, 10);
+    if (bytes > lim)
+        return fail(ISV_ENOMEM_PINNED,
+                    "pinned allocation of %llu bytes for the host KV pool refused: ISV_PINNED_LIMIT_BYTES is %llu "
+                    "(fewer phys_layers or a smaller offload_frac need less)",
+                    (unsigned long long)bytes, lim);
+    return ISV_OK;
+}
+
 int check_handle(isv_kv *h, int layer, bool need_device) {
     if (!h) return fail(ISV_EINVAL, "null handle");
     if (layer < 0 || layer >= h->g.layers) return fail(ISV_EINVAL, "layer %d out of range [0, %d)", layer, h->g.layers);
@@ -205,6 +225,31 @@ int check_handle(isv_kv *h, int layer, bool need_device) {
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Host-side wait for a stream.  Without a limit it blocks in the driver; with one (isv_set_host_timeout)
+// it polls and returns ISV_ETIMEOUT when the deadline passes, leaving the work enqueued.
+int wait_stream(isv_kv *h, cudaStream_t st, const char *what) {
+    if (!st) return ISV_OK;
+    if (h->host_timeout_s <= 0.0) {
+        CU(cudaStreamSynchronize(st));
+        return ISV_OK;
+    }
+    const auto deadline = std::chrono::steady_clock::now() + std::chrono::duration<double>(h->host_timeout_s);
+    for (;;) {
+        const cudaError_t e = cudaStreamQuery(st);
+        if (e == cudaSuccess) return ISV_OK;
+        if (e != cudaErrorNotReady) return fail(ISV_ECUDA, "cudaStreamQuery(%s): %s", what, cudaGetErrorString(e));
+        if (std::chrono::steady_clock::now() >= deadline)
+            return fail(ISV_ETIMEOUT, "the %s stream did not finish within %.3f s (work is still enqueued)", what,
+                        h->host_timeout_s);
+        std::this_thread::sleep_for(std::chrono::microseconds(50));
+    }
+}
+#define WAIT(stream, what)                                   \
+    do {                                                     \
+        const int rc_ = wait_stream(h, (stream), (what));    \
+        if (rc_) return rc_;                                 \
+    } while (0)
 
 // Pushes table updates to the device copy, kMaxTableUpdates per launch (by value).
 int push_updates(isv_kv *h, const std::vector<TableUpdate> &upd) {
@@ -350,7 +395,12 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
     h->g = g;
     h->plan_only = desc->plan_only != 0;
     h->bm.init(g, desc->perm_seed);
-    if (h->plan_only) { *out = h; return ISV_OK; }
+    if (h->plan_only) {   // a plan tells whether the host pool would be accepted, without allocating it
+        const int rc_lim = check_pinned_limit((uint64_t)g.phys_layers * g.host_cap * g.block_bytes);
+        if (rc_lim) { delete h; return rc_lim; }
+        *out = h;
+        return ISV_OK;
+    }
 
     int rc = ISV_OK;
     auto bail = [&](int code) { destroy(h); return code; };
@@ -393,6 +443,7 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
         const size_t tail_bytes = (size_t)g.phys_layers * g.max_seqs * g.block_bytes;
         if ((rc = dev_alloc((void **)&h->tail, tail_bytes, &h->hbm_pool_bytes, "tail slots"))) return bail(rc);
         h->host_pool_bytes = (uint64_t)g.phys_layers * g.host_cap * g.block_bytes;
+        if ((rc = check_pinned_limit(h->host_pool_bytes))) return bail(rc);
         cudaError_t e = cudaHostAlloc((void **)&h->pool_host, h->host_pool_bytes,
                                       cudaHostAllocMapped | cudaHostAllocPortable);
         if (e != cudaSuccess) {
@@ -469,11 +520,11 @@ int isv_sync(isv_kv *h, uint32_t *status_out) {
     if (!h) return fail(ISV_EINVAL, "null handle");
     if (status_out) *status_out = 0;
     if (h->plan_only) return ISV_OK;
-    CU(cudaStreamSynchronize(h->s_compute));
-    CU(cudaStreamSynchronize(h->s_copy));
-    CU(cudaStreamSynchronize(h->s_off));
-    CU(cudaStreamSynchronize(h->s_d2h));
-    if (h->s_in) CU(cudaStreamSynchronize(h->s_in));
+    WAIT(h->s_compute, "compute");
+    WAIT(h->s_copy, "copy");
+    WAIT(h->s_off, "offloaded-attention");
+    WAIT(h->s_d2h, "write-back");
+    WAIT(h->s_in, "step-input");
     uint32_t st = 0;
     CU(cudaMemcpy(&st, h->status_dev, 4, cudaMemcpyDeviceToHost));
     if (status_out) *status_out = st;
@@ -481,9 +532,10 @@ int isv_sync(isv_kv *h, uint32_t *status_out) {
         CU(cudaMemset(h->status_dev, 0, 4));
         // a kernel that gave up may have left its arrival counters half way
         CU(cudaMemset(h->tickets, 0, (size_t)h->g.max_seqs * h->g.Hkv * h->g.P * 4));
-        return fail(ISV_EDEVICE_STATUS, "a kernel reported status 0x%x (%s%s)", st,
+        return fail(ISV_EDEVICE_STATUS, "a kernel reported status 0x%x (%s%s%s)", st,
                     (st & ISV_STATUS_BAD_BLOCK_ID) ? "bad block id " : "",
-                    (st & ISV_STATUS_WAIT_EXPIRED) ? "wait expired" : "");
+                    (st & ISV_STATUS_WAIT_EXPIRED) ? "wait expired " : "",
+                    (st & ISV_STATUS_BAD_LENGTH) ? "bad length" : "");
     }
     return ISV_OK;
 }
@@ -548,7 +600,7 @@ int isv_kv_fill_async(isv_kv *h, int32_t layer, const void *k, const void *v, co
     if (h->plan_only) return ISV_OK;
 
     // the table and lengths are replaced wholesale: earlier kernels must be done with them
-    CU(cudaStreamSynchronize(h->s_compute));
+    WAIT(h->s_compute, "compute");
     CU(cudaMemcpy(h->table_dev, h->bm.table.data(), h->bm.table.size() * 4, cudaMemcpyHostToDevice));
     CU(cudaMemcpy(lens_ptr(h, layer, 0), &h->bm.len[(size_t)layer * g.max_seqs],
                   (size_t)g.max_seqs * 4, cudaMemcpyHostToDevice));
@@ -654,8 +706,8 @@ int isv_kv_fill(isv_kv *h, int32_t layer, const void *k, const void *v, const in
                 int32_t n_seqs, int32_t T) {
     int rc = isv_kv_fill_async(h, layer, k, v, lens_host, n_seqs, T);
     if (rc || h->plan_only) return rc;
-    CU(cudaStreamSynchronize(h->s_compute));
-    CU(cudaStreamSynchronize(h->s_d2h));
+    WAIT(h->s_compute, "compute");
+    WAIT(h->s_d2h, "write-back");
     return ISV_OK;
 }
 
@@ -664,8 +716,8 @@ int isv_fill_timing(isv_kv *h, isv_fill_times *out) {
     if (h->plan_only) return fail(ISV_ENODEVICE, "plan-only handle");
     memset(out, 0, sizeof *out);
     if (!h->fill_timed) return ISV_OK;
-    CU(cudaStreamSynchronize(h->s_compute));
-    CU(cudaStreamSynchronize(h->s_d2h));
+    WAIT(h->s_compute, "compute");
+    WAIT(h->s_d2h, "write-back");
     float t = 0.f;
     if (cudaEventElapsedTime(&t, h->ev_f0, h->ev_f1) == cudaSuccess) out->pack_ms = t;
     out->total_ms = out->pack_ms;
@@ -706,7 +758,7 @@ int isv_kv_append(isv_kv *h, int32_t layer, const void *k, const void *v, int32_
     p.table = h->table_dev;
     p.lens = lens_ptr(h, layer, 0);
     p.status = h->status_dev;
-    p.table_stride = g.NB; p.n_pool_blocks = g.hbm_cap;
+    p.table_stride = g.NB; p.n_pool_blocks = g.hbm_cap; p.max_blocks = g.NB;
     p.n_seqs = n_seqs; p.Hkv = g.Hkv; p.D = g.D; p.BT = g.BT;
     p.block_bytes = g.block_bytes;
     CU(launch_append(p, h->s_compute));
@@ -756,6 +808,8 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
     base.table = block_table_dev ? block_table_dev : h->table_dev;
     base.lens = seq_lens_dev ? seq_lens_dev : lens_ptr(h, layer, 0);
     base.table_stride = g.NB;
+    base.max_blocks = g.NB;
+    base.spin_limit = h->spin_limit;
     base.q = q;
     base.status = h->status_dev;
     base.n_seqs = n_seqs; base.Hq = g.Hq; base.Hkv = g.Hkv; base.P = g.P; base.GT = g.GT;
@@ -853,6 +907,10 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
             nu += (long long)std::max(1, (h->bm.length(layer, s) + g.BT - 1) / g.BT) * Hg;
         const int cap = g.max_ctas > 0 ? std::min(g.max_ctas, h->sm_count) : h->sm_count;
         const int grid = (int)std::max<long long>(1, std::min<long long>(cap, (nu + nw - 1) / nw));
+        if (h->lost_copies > 0) {
+            --h->lost_copies;
+            p.drop_first_copy = 1;
+        }
         if (le) CU(cudaEventRecord(le->r0, h->s_compute));
         CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_RESIDENT, grid, h->stages_res, h->smem_res, h->s_compute));
         ++h->launches;
@@ -906,16 +964,19 @@ int isv_decode_layer(isv_kv *h, int32_t layer, const void *q, const void *k, con
     return flush_tails(h, layer, ap.flush);
 }
 
-int isv_decode_step(isv_kv *h, const void *q, const void *k, const void *v, void *out, int32_t n_seqs) {
+int isv_decode_step(isv_kv *h, const void *q, const void *k, const void *v, void *out, float *out_f32,
+                    int32_t n_seqs) {
     int rc = check_handle(h, 0, true);
     if (rc) return rc;
     const Geometry &g = h->g;
-    if (!q || !k || !v || !out) return fail(ISV_EINVAL, "q, k, v and out must be given");
+    if (!q || !k || !v || (!out && !out_f32)) return fail(ISV_EINVAL, "q, k, v and one of out / out_f32 must be given");
     if (n_seqs < 0 || n_seqs > g.max_seqs) return fail(ISV_EINVAL, "n_seqs %d outside [0, %d]", n_seqs, g.max_seqs);
-    const size_t qs = (size_t)n_seqs * g.Hq * g.D * 2, ks = (size_t)n_seqs * g.Hkv * g.D * 2;
+    const size_t rows = (size_t)n_seqs * g.Hq * g.D;
+    const size_t qs = rows * 2, ks = (size_t)n_seqs * g.Hkv * g.D * 2;
     for (int l = 0; l < g.layers; ++l) {
         if ((rc = isv_decode_layer(h, l, (const uint8_t *)q + l * qs, (const uint8_t *)k + l * ks,
-                                   (const uint8_t *)v + l * ks, (uint8_t *)out + l * qs, nullptr, n_seqs)))
+                                   (const uint8_t *)v + l * ks, out ? (uint8_t *)out + l * qs : nullptr,
+                                   out_f32 ? out_f32 + l * rows : nullptr, n_seqs)))
             return rc;
     }
     return ISV_OK;
@@ -979,8 +1040,8 @@ int isv_decode_step_host(isv_kv *h, const void *q, const void *k, const void *v,
         CU(cudaStreamWaitEvent(h->s_d2h, h->ev_step_out[gi], 0));
         CU(cudaMemcpyAsync((uint8_t *)out + l0 * ql, dout + l0 * ql, nl * ql, cudaMemcpyDeviceToHost, h->s_d2h));
     }
-    CU(cudaStreamSynchronize(h->s_compute));
-    CU(cudaStreamSynchronize(h->s_d2h));
+    WAIT(h->s_compute, "compute");
+    WAIT(h->s_d2h, "write-back");
     return ISV_OK;
 }
 
@@ -1008,7 +1069,10 @@ int isv_kv_gather(isv_kv *h, int32_t layer, int32_t seq, void *k_host, void *v_h
     h->last_fused_layer = -1;
     cudaError_t e = launch_gather(p, h->s_compute);
     ++h->launches;
-    if (e == cudaSuccess) e = cudaStreamSynchronize(h->s_compute);
+    if (e == cudaSuccess && (rc = wait_stream(h, h->s_compute, "compute"))) {
+        cudaFree(tmp);
+        return rc;
+    }
     if (e == cudaSuccess) e = cudaMemcpy(k_host, tmp, bytes, cudaMemcpyDeviceToHost);
     if (e == cudaSuccess) e = cudaMemcpy(v_host, tmp + bytes, bytes, cudaMemcpyDeviceToHost);
     cudaFree(tmp);
@@ -1062,6 +1126,26 @@ int isv_plan_bytes(isv_kv *h, int32_t layer, int32_t n_seqs, uint64_t *res, uint
 int isv_set_zero_copy(isv_kv *h, int32_t on) {
     if (!h) return fail(ISV_EINVAL, "null handle");
     h->zero_copy = on != 0;
+    return ISV_OK;
+}
+
+int isv_set_host_timeout(isv_kv *h, double seconds) {
+    if (!h) return fail(ISV_EINVAL, "null handle");
+    if (!(seconds >= 0.0)) return fail(ISV_EINVAL, "the timeout must be >= 0 seconds (0 = none)");
+    h->host_timeout_s = seconds;
+    return ISV_OK;
+}
+
+int isv_set_wait_limit(isv_kv *h, uint32_t polls) {
+    if (!h) return fail(ISV_EINVAL, "null handle");
+    h->spin_limit = polls;
+    return ISV_OK;
+}
+
+int isv_inject_lost_copy(isv_kv *h, int32_t launches) {
+    if (!h) return fail(ISV_EINVAL, "null handle");
+    if (launches < 0) return fail(ISV_EINVAL, "launches must be >= 0");
+    h->lost_copies = launches;
     return ISV_OK;
 }
 

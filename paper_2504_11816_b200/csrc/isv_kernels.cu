@@ -19,7 +19,7 @@ namespace {
 
 constexpr float kNegBig = -1.0e30f;          // "no score yet": finite so differences never give NaN
 constexpr uint32_t kFull = 0xffffffffu;
-constexpr uint32_t kSpinLimit = 1u << 22;    // polls before a wait gives up
+constexpr uint32_t kSpinLimit = 1u << 22;    // polls before a wait gives up (DecodeParams::spin_limit overrides it)
 
 // ---------------------------------------------------------------- PTX helpers
 
@@ -52,9 +52,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the phase did not complete within kSpinLimit polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+// Bounded wait: false when the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 256) __nanosleep(64);
     }
@@ -134,9 +134,18 @@ __device__ __forceinline__ int swz(int chunk, int t, int nchunks) {
 // 64-element span v.  Each group keeps its own running (m, l, o); groups are merged at unit end.
 // head_dim 80 leaves a tail of 16 elements = 2 chunks per token.  Giving it to lanes sub 0 and 1 of every
 // pass would cost a whole span's instructions for a quarter of the lanes, so the tails of a group's four
-// tokens are handled in one extra step instead: lane sub takes the tail chunk (sub & 1) of the token of
-// pass sub / 2.  Its registers q[.][NVF*8 ..] / o[.][NVF*8 ..] then belong to elements
+// tokens are handled in one extra step instead: lane sub takes the tail chunk (sub & 1) of one token of
+// pass sub / 2 (for K: tail_token below; for V: the group's own token of that pass).  Its registers q[.][NVF*8 ..] / o[.][NVF*8 ..] then belong to elements
 // NVF*64 + (sub & 1)*8 .., and the o tails of the lanes with equal sub & 1 are summed at unit end.
+
+// Token whose 16-element K tail lane (grp, sub) handles: that of pass pi = sub / 2 of group (grp + pi) mod 4.
+// The rotation by pi makes the four tokens one quarter-warp reads differ mod 4, so its eight 16-byte loads
+// (rows are 160 bytes apart) fall into eight different bank groups instead of colliding four ways.  Scores
+// are plain numbers and travel back to the owning group by a shuffle.
+__device__ __forceinline__ int tail_token(int grp, int sub) {
+    const int pi = sub >> 1;
+    return 4 * pi + ((grp + pi) & 3);
+}
 
 // Scores of the tile's tokens against the GT query heads (log2 domain, q is
 // pre-scaled), and the running maximum brought up to date (o and l rescaled).
@@ -172,8 +181,8 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
             sc[i][g] = a;
         }
     }
-    if (NV > NVF) {   // the 16-element tails of the group's four tokens, one chunk per lane
-        const int tt = 4 * (sub >> 1) + grp;
+    if (NV > NVF) {   // the 16-element tails, one chunk per lane (token assignment: see tail_token)
+        const int tt = tail_token(grp, sub);
         float kf[8];
         cvt8<BF16>(reinterpret_cast<const uint4 *>(sK + tt * ROW)[NVF * 8 + (sub & 1)], kf);
 #pragma unroll
@@ -181,9 +190,10 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
             float tp = 0.f;
 #pragma unroll
             for (int e = 0; e < 8; ++e) tp = fmaf(q[g][NVF * 8 + e], kf[e], tp);
-            tp += __shfl_xor_sync(kFull, tp, 1);   // lanes 2i and 2i+1 of the group: tail of the token of pass i
+            tp += __shfl_xor_sync(kFull, tp, 1);   // lanes 2i and 2i+1 of a group: the two tail chunks of one token
 #pragma unroll
-            for (int i = 0; i < NQ; ++i) sc[i][g] += __shfl_sync(kFull, tp, grp * 8 + 2 * i);
+            for (int i = 0; i < NQ; ++i)   // the tail of this group's token of pass i was taken by group (grp - i) mod 4
+                sc[i][g] += __shfl_sync(kFull, tp, ((grp - i) & 3) * 8 + 2 * i);
         }
     }
 #pragma unroll
@@ -239,6 +249,8 @@ __device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp
         }
     }
     if (NV > NVF) {
+        // The V tails stay with the group that owns the token: their products are added to that group's
+        // accumulators, which are scaled by that group's running maximum (no rotation as for the K tails).
         const int pi = sub >> 1, tt = 4 * pi + grp;
         if (tt < ntok) {
             float vf[8];
@@ -947,15 +959,22 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * (8 + 4 * V_WORDS));   // [n_seqs + 1]
     int32_t *slen = ubase + p.n_seqs + 1;   // [n_seqs] tokens to attend (resident mode)
 
-    // Programmatic dependent launch: let the next kernel in the stream begin its launch as this one's
-    // CTAs retire, and do not read anything an earlier kernel may have written before that kernel is done.
-    // With early_reads the wait is postponed until after the first K/V copies are issued: lengths, block
-    // table and this layer's KV slab were last written by kernels that finished long ago (only the kernel
-    // launched immediately before may still be running, and the host sets the flag only when that kernel
-    // writes none of them), whereas q, the new K/V rows, the scratch and the outputs are touched only
-    // after the wait.  The pipeline's ramp-up then overlaps the previous kernel's tail.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (!p.early_reads) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Programmatic dependent launch.  This kernel may start while its predecessor in the stream is
+    // still running; griddepcontrol.wait returns once that predecessor has completed and its writes
+    // are visible, and only after its own wait does a CTA let the successor start
+    // (griddepcontrol.launch_dependents).  The order matters: a successor begins once every CTA of
+    // this grid has released it, so at that moment the predecessor of this grid is complete, and by
+    // induction at most two kernels of a chain are ever in flight, whatever the grid sizes.
+    // With early_reads the wait is postponed until after the first K/V copies are issued: the host
+    // sets the flag only when the immediate predecessor writes neither the lengths, nor the block
+    // table, nor this layer's KV slab, and every kernel before that one has completed by the time
+    // this one starts; q, the new K/V rows, the scratch and the outputs are touched only after the
+    // wait.  The pipeline's ramp-up then overlaps the predecessor's tail.
+    if (!p.early_reads) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
+    const uint32_t spin_limit = p.spin_limit ? p.spin_limit : kSpinLimit;
 
     const int Hg = p.Hkv * p.P;
     const uint64_t block_bytes = p.block_bytes;
@@ -968,8 +987,12 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     // Staged mode: whole (chunk unit, head group) items.
     long long NU;
     if (MODE == MODE_RESIDENT) {
+        const int len_cap = p.max_blocks * BT;
         for (int s = threadIdx.x; s < p.n_seqs; s += blockDim.x) {
-            const int len = p.lens[s] + fused;
+            // a length the table row does not cover is never followed into the table
+            const int raw = p.lens[s];
+            const int len = min(max(raw, 0) + fused, len_cap);
+            if (len != raw + fused) atomicOr(p.status, ISV_STATUS_BAD_LENGTH);
             slen[s] = len;
             ubase[s + 1] = max(1, (len + BT - 1) / BT) * Hg;
         }
@@ -1022,6 +1045,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     bool pu_open = false, pu_done = false;
     const uint8_t *pv_src = nullptr;    // V tile of the visit whose K slot was armed last (NULL: no tiles)
     int prod_vis = 0, inflight = 0;     // ring position of the next visit to emit; visits emitted and not consumed
+    bool drop_copy = p.drop_first_copy && blockIdx.x == 0 && warp == 0;   // failure injection, see DecodeParams
     if (MODE == MODE_RESIDENT) {   // sequence of the first unit: largest s with ubase[s] <= u_next
         int lo = 0, hi = p.n_seqs - 1;
         while (lo < hi) {
@@ -1152,7 +1176,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             const uint32_t bar = smem_u32(&bars[2 * prod_vis]);
             if (ksrc) {
                 mbar_arrive_expect_tx(bar, TILE);
-                bulk_g2s(smem_u32(data + (size_t)(2 * prod_vis) * TILE), ksrc, TILE, bar);
+                if (!drop_copy) bulk_g2s(smem_u32(data + (size_t)(2 * prod_vis) * TILE), ksrc, TILE, bar);
+                drop_copy = false;
             } else {
                 mbar_arrive(bar);
             }
@@ -1179,7 +1204,10 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             if (!produce_k()) break;
             produce_v();
         }
-    if (p.early_reads) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (p.early_reads) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
 
     // ---- fused append (placed after the first copies are in flight so that it costs no start-up time):
     // the rows of this step's token go to slot len % BT of block len / BT
@@ -1227,7 +1255,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         if (lane == 0)
             asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
                          : "=r"(ticket) : "l"(&p.tickets[pend.ticket_idx]) : "memory");
-        ticket = __shfl_sync(kFull, ticket, 0);   // the other lanes read the partials after lane 0's acquire
+        ticket = __shfl_sync(kFull, ticket, 0);
+        __syncwarp();   // orders the other lanes' reads of the partials after lane 0's acquire
         if (ticket == pend.nc - 1) {
             if (lane == 0) p.tickets[pend.ticket_idx] = 0;   // ready for the next launch
             if (at_end && GT > 1) {   // the accumulators are dead: several heads at a time
@@ -1249,14 +1278,14 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     auto give_up = [&]() {
         if (lane == 0) atomicOr(p.status, ISV_STATUS_WAIT_EXPIRED);
         for (int k = 0; k < inflight; ++k) {
-            mbar_wait(smem_u32(&bars[2 * cons_vis]), cons_phase);
-            mbar_wait(smem_u32(&bars[2 * cons_vis + 1]), cons_phase);
+            mbar_wait(smem_u32(&bars[2 * cons_vis]), cons_phase, spin_limit);
+            mbar_wait(smem_u32(&bars[2 * cons_vis + 1]), cons_phase, spin_limit);
             cons_vis = (cons_vis + 1 == NVIS) ? 0 : cons_vis + 1;
             if (cons_vis == 0) cons_phase ^= 1u;
         }
     };
     while (inflight > 0) {
-        bool ok = mbar_wait(smem_u32(&bars[2 * cons_vis]), cons_phase);
+        bool ok = mbar_wait(smem_u32(&bars[2 * cons_vis]), cons_phase, spin_limit);
         if (!__all_sync(kFull, ok)) {
             give_up();
             return;
@@ -1279,7 +1308,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         __syncwarp();   // every lane is done with the K slot and the record before they are refilled
         const bool more = !pu_done && produce_k();
 
-        ok = mbar_wait(smem_u32(&bars[2 * cons_vis + 1]), cons_phase);
+        ok = mbar_wait(smem_u32(&bars[2 * cons_vis + 1]), cons_phase, spin_limit);
         if (!__all_sync(kFull, ok)) {
             give_up();
             return;
@@ -1376,7 +1405,8 @@ __global__ void append_kernel(const AppendParams p) {
     const int s = blockIdx.x;
     const int len = p.lens[s];
     const int j = len / p.BT, slot = len % p.BT;
-    const int32_t e = p.table[(size_t)s * p.table_stride + j];
+    const bool in_row = len >= 0 && j < p.max_blocks;   // a length the table row does not cover is not followed
+    const int32_t e = in_row ? p.table[(size_t)s * p.table_stride + j] : ISV_BLOCK_NONE;
     uint8_t *base = nullptr;
     if (e != ISV_BLOCK_NONE) {
         if (e & ISV_BLOCK_HOST_BIT) {
@@ -1401,10 +1431,10 @@ __global__ void append_kernel(const AppendParams p) {
             *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
         }
     } else if (threadIdx.x == 0) {
-        atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
+        atomicOr(p.status, in_row ? ISV_STATUS_BAD_BLOCK_ID : ISV_STATUS_BAD_LENGTH);
     }
     __syncthreads();   // every thread has read the old length
-    if (threadIdx.x == 0) p.lens[s] = len + 1;
+    if (threadIdx.x == 0 && in_row) p.lens[s] = len + 1;
 }
 
 // Where block j of sequence s lives for a reader/writer that sees `len`

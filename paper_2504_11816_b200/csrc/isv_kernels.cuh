@@ -29,6 +29,8 @@ struct DecodeParams {
     const int32_t *table;       // [n_seqs][table_stride]
     const int32_t *lens;        // [n_seqs] tokens to attend
     int32_t table_stride;
+    int32_t max_blocks;         // resident: table entries of a row that may be read; lengths beyond
+                                // max_blocks * BT tokens (or negative) are clamped and flagged
     int32_t n_pool_blocks;      // bound for block ids (pool blocks, or slots in the staging buffer)
     // staged mode lists
     const int32_t *cu_seq;
@@ -58,6 +60,9 @@ struct DecodeParams {
     int32_t GT;                 // query heads of one head group (Hq = Hkv * P * GT)
     int32_t finalize;           // resident: 1 = normalise and write out; 0 = leave (m, l, o) in acc_*
     int32_t early_reads;        // 1 = lengths, table and KV may be read before the dependency wait
+    uint32_t spin_limit;        // polls after which a wait on a copy gives up (0 = default)
+    int32_t drop_first_copy;    // failure injection: warp 0 of CTA 0 arms its first K slot without issuing
+                                // the copy, as if the transfer had been lost (its wait then runs out)
     float scale_log2;           // log2(e) / sqrt(D)
     uint64_t block_bytes;
 };
@@ -76,6 +81,7 @@ struct AppendParams {
     int32_t *lens;              // [n_seqs], incremented by the kernel
     uint32_t *status;
     int32_t table_stride, n_pool_blocks;
+    int32_t max_blocks;         // table entries of a row that may be read (a full sequence is flagged)
     int32_t n_seqs, Hkv, D, BT;
     uint64_t block_bytes;
 };

@@ -163,6 +163,7 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     p.table = block_table_dev;
     p.lens = seq_lens_dev;
     p.table_stride = table_stride;
+    p.max_blocks = max_blocks_per_seq;      // longer (or negative) lengths are clamped and flagged
     p.n_pool_blocks = n_pool_blocks;
     p.q = q_dev;
     p.out = out_dev;

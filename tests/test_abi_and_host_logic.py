@@ -179,3 +179,37 @@ def test_pool_sizes_follow_the_kv_size_formula():
         assert info.hbm_pool_bytes == pm.kv_cache_bytes(32, 1152, 2560, 2, 32)
     finally:
         B.isv_kv_free(h)
+
+
+def test_host_pool_beyond_the_pinned_limit_is_refused(monkeypatch):
+    """ISV_PINNED_LIMIT_BYTES stands in for a locked-memory limit of the system: a description whose
+    host pool exceeds it is refused with ISV_ENOMEM_PINNED and a message, on plan-only handles too."""
+    need = B.isv_kv_info(h0 := _alloc()).host_pool_bytes
+    B.isv_kv_free(h0)
+    assert need > 0
+    monkeypatch.setenv("ISV_PINNED_LIMIT_BYTES", str(need - 1))
+    with pytest.raises(B.IsvError) as ei:
+        _alloc()
+    assert ei.value.code == B.ISV_ENOMEM_PINNED
+    assert str(need) in ei.value.message and "ISV_PINNED_LIMIT_BYTES" in ei.value.message
+    monkeypatch.setenv("ISV_PINNED_LIMIT_BYTES", str(need))
+    B.isv_kv_free(_alloc())
+    B.isv_kv_free(_alloc(offload_frac=0.0))          # nothing offloaded: no host pool, never refused
+
+
+def test_failure_handling_knobs_validate_their_arguments():
+    h = _alloc()
+    try:
+        B.isv_set_host_timeout(h, 2.5)
+        B.isv_set_host_timeout(h, 0.0)
+        with pytest.raises(B.IsvError) as ei:
+            B.isv_set_host_timeout(h, -1.0)
+        assert ei.value.code == B.ISV_EINVAL
+        B.isv_set_wait_limit(h, 1000)
+        B.isv_inject_lost_copy(h, 0)
+        with pytest.raises(B.IsvError) as ei:
+            B.isv_inject_lost_copy(h, -1)
+        assert ei.value.code == B.ISV_EINVAL
+        assert B.isv_sync(h) == 0                    # a plan-only handle has nothing to wait for
+    finally:
+        B.isv_kv_free(h)

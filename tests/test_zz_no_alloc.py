@@ -48,7 +48,10 @@ def _paged_pool(k_bits, v_bits, lens, kv_heads, head_dim, seed):
     return pool, table, total, stride, max(nb)
 
 
-@pytest.mark.parametrize("q_heads,kv_heads,head_dim,dtype", [(8, 8, 128, "f16"), (8, 2, 64, "bf16"), (4, 4, 80, "f16")])
+# the last shape (16 query heads per KV head at head_dim 128) needs 133 KB of partials per CTA: a full grid
+# does not fit the fixed array, so the call runs on the 62 CTAs whose partials do
+@pytest.mark.parametrize("q_heads,kv_heads,head_dim,dtype", [(8, 8, 128, "f16"), (8, 2, 64, "bf16"), (4, 4, 80, "f16"),
+                                                             (32, 2, 128, "f16")])
 def test_static_entry_matches_handle_entry_on_two_calls_in_a_row(q_heads, kv_heads, head_dim, dtype):
     lens = [300, 1, 16, 513, 77]
     w = W.Workload("na", 1, q_heads, kv_heads, head_dim, dtype, len(lens), 1, 513, 2, 16, 0.0, 0, 31)
