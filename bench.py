@@ -456,10 +456,15 @@ def measure_point(cx: Ctx, w, K, Wm, reps, reset_between, want_e2e, phys_req=0):
         res_bytes_launch = last_step.bytes_resident / w.layers
         timed = "CUDA events around every launch of the last timed step (a launch lasts far longer than an event gap)"
     else:
-        avg_ms = ms / n_launch
-        res_bytes_launch = per_ls_res
-        timed = ("CUDA events around the timed region / launches in it (one decode_kernel launch per layer-step; "
-                 "includes the gaps between launches)")
+        # nothing offloaded: the region holds decode_kernel launches and nothing else (bar a table update every
+        # 16 steps) - one per step covering all layers, or one per layer-step where that is switched off
+        whole_step = med["launches"] < n_launch
+        dec_launches = K if whole_step else n_launch
+        avg_ms = ms / dec_launches
+        res_bytes_launch = med["bytes_res"] / dec_launches
+        timed = ("CUDA events around the timed region / decode_kernel launches in it (one launch per "
+                 + ("step, covering all layers" if whole_step else "layer-step")
+                 + "; includes the gaps between launches)")
     achieved = res_bytes_launch / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else 0.0
     traffic = None
     if NCU_TRAFFIC["kernels_sha1"] == kernels_sha1():   # counters taken from this very kernel source

@@ -104,6 +104,7 @@ struct isv_kv {
     // kernel configuration
     int stages_res = 0, stages_stg = 0;
     size_t smem_res = 0, smem_stg = 0;
+    int smem_limit = 0;                    // opt-in shared memory per block of the device
     uint64_t launches = 0;                 // kernels launched so far
     int last_fused_layer = -1;             // layer of the latest fused decode launch if nothing else of ours
                                            // was launched on the compute stream since, else -1
@@ -125,6 +126,8 @@ int32_t *lens_ptr(const isv_kv *h, int layer, int which) {
     const int copy = (h->lens_cur[layer] ^ which) & 1;
     return h->lens_dev + ((size_t)copy * h->g.layers + layer) * h->g.max_seqs;
 }
+
+size_t tickets_bytes(const Geometry &g) { return (size_t)g.layers * g.max_seqs * g.Hkv * g.P * 4; }
 
 size_t slab_hbm(const isv_kv *h, int layer) {
     return (size_t)(layer % h->g.phys_layers) * h->g.hbm_cap * h->g.block_bytes;
@@ -417,6 +420,7 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
     if (prop.major < 9)
         return bail(fail(ISV_ECUDA, "device compute capability %d.%d lacks bulk async copies", prop.major, prop.minor));
     const int smem_limit = (int)prop.sharedMemPerBlockOptin;
+    h->smem_limit = smem_limit;
     h->stages_res = pick_stages(g, MODE_RESIDENT, smem_limit, &h->smem_res);
     h->stages_stg = pick_stages(g, MODE_STAGED, smem_limit, &h->smem_stg);
     if (h->stages_res < 2 || h->stages_stg < 2)
@@ -470,8 +474,9 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
     const size_t slots = 2ull * max_grid * decode_warps(g.GT, g.D) * g.GT;   // two partials per warp and query head
     if ((rc = dev_alloc((void **)&h->part_o, slots * g.D * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
     if ((rc = dev_alloc((void **)&h->part_ml, slots * 2 * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
-    if ((rc = dev_alloc((void **)&h->tickets, (size_t)g.max_seqs * g.Hkv * g.P * 4, &h->scratch_bytes, "tickets"))) return bail(rc);
-    CUB(cudaMemset(h->tickets, 0, (size_t)g.max_seqs * g.Hkv * g.P * 4));
+    // one arrival counter per (layer, sequence, head group): a launch that covers several layers uses them all
+    if ((rc = dev_alloc((void **)&h->tickets, tickets_bytes(g), &h->scratch_bytes, "tickets"))) return bail(rc);
+    CUB(cudaMemset(h->tickets, 0, tickets_bytes(g)));
     if (g.host_cap > 0) {
         if ((rc = dev_alloc((void **)&h->res_o, rows * g.D * 4, &h->scratch_bytes, "resident result"))) return bail(rc);
         if ((rc = dev_alloc((void **)&h->res_ml, rows * 2 * 4, &h->scratch_bytes, "resident result"))) return bail(rc);
@@ -531,7 +536,7 @@ int isv_sync(isv_kv *h, uint32_t *status_out) {
     if (st != 0) {
         CU(cudaMemset(h->status_dev, 0, 4));
         // a kernel that gave up may have left its arrival counters half way
-        CU(cudaMemset(h->tickets, 0, (size_t)h->g.max_seqs * h->g.Hkv * h->g.P * 4));
+        CU(cudaMemset(h->tickets, 0, tickets_bytes(h->g)));
         return fail(ISV_EDEVICE_STATUS, "a kernel reported status 0x%x (%s%s%s)", st,
                     (st & ISV_STATUS_BAD_BLOCK_ID) ? "bad block id " : "",
                     (st & ISV_STATUS_WAIT_EXPIRED) ? "wait expired " : "",
@@ -547,7 +552,7 @@ int isv_kv_reset(isv_kv *h) {
         if (rc && rc != ISV_EDEVICE_STATUS) return rc;
         CU(cudaMemset(h->table_dev, 0xff, (size_t)h->g.max_seqs * h->g.NB * 4));
         CU(cudaMemset(h->lens_dev, 0, 2 * (size_t)h->g.layers * h->g.max_seqs * 4));
-        CU(cudaMemset(h->tickets, 0, (size_t)h->g.max_seqs * h->g.Hkv * h->g.P * 4));
+        CU(cudaMemset(h->tickets, 0, tickets_bytes(h->g)));
         std::fill(h->flush_recorded.begin(), h->flush_recorded.end(), 0);
         h->owner_uploaded = -1;
         h->last_fused_layer = -1;
@@ -964,6 +969,83 @@ int isv_decode_layer(isv_kv *h, int32_t layer, const void *q, const void *k, con
     return flush_tails(h, layer, ap.flush);
 }
 
+// Whether layers [l0, l0 + nl) of a step can run as one launch: nothing of the cache is offloaded (no
+// staging, no tail slots, no per-layer merge), per-layer timing is off (there is no per-layer launch to
+// time), and the kernel's per-(layer, sequence) tables fit in shared memory beside the full ring.
+static bool can_fuse_layers(const isv_kv *h, int nl, int n_seqs, size_t *smem) {
+    const Geometry &g = h->g;
+    if (nl < 2 || n_seqs < 1 || h->timing || g.host_cap != 0 || g.layers > 64) return false;
+    if (const char *e = getenv("ISV_LAYERS_PER_LAUNCH"))   // tuning knob: 1 = one launch per layer
+        if (atoi(e) == 1) return false;
+    const size_t b = decode_smem_bytes(g.D, g.BT, g.GT, h->stages_res, nl * n_seqs, MODE_RESIDENT);
+    if (b > (size_t)h->smem_limit) return false;
+    *smem = b;
+    return true;
+}
+
+// Layers [l0, l0 + nl) of one decode step (append + attention each) as ONE launch of the resident kernel.
+// q, out, out_f32: [nl][n_seqs][q_heads][head_dim]; k, v: [nl][n_seqs][kv_heads][head_dim], device.
+static int decode_layers_fused(isv_kv *h, int l0, int nl, const void *q, const void *k, const void *v, void *out,
+                               float *out_f32, int n_seqs, size_t smem) {
+    const Geometry &g = h->g;
+    int rc = ISV_OK;
+    // host side of the appends; nothing stays changed when a layer cannot take its token
+    for (int l = l0; l < l0 + nl; ++l)
+        for (int s = 0; s < n_seqs; ++s)
+            if (h->bm.length(l, s) >= g.max_tokens)
+                return fail(ISV_ECAPACITY, "sequence %d is full (%d tokens)", s, h->bm.length(l, s));
+    AppendPlan ap;
+    for (int l = l0; l < l0 + nl; ++l) {
+        if ((rc = append_bookkeeping(h, l, n_seqs, &ap))) {
+            for (int lb = l0; lb < l; ++lb)
+                for (int s = 0; s < n_seqs; ++s) --h->bm.length(lb, s);
+            push_updates(h, ap.upd);   // blocks handed out so far stay allocated
+            return rc;
+        }
+    }
+    if ((rc = push_updates(h, ap.upd))) return rc;
+
+    const bool bf16 = g.dtype == ISV_BF16;
+    const int Hg = g.Hkv * g.P;
+    const int nw = decode_warps(g.GT, g.D);
+    DecodeParams p{};
+    p.table = h->table_dev;
+    p.table_stride = g.NB;
+    p.max_blocks = g.NB;
+    p.spin_limit = h->spin_limit;
+    p.status = h->status_dev;
+    p.n_seqs = n_seqs; p.Hq = g.Hq; p.Hkv = g.Hkv; p.P = g.P; p.GT = g.GT;
+    p.block_bytes = g.block_bytes;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)g.D));
+    p.pool = h->pool_hbm; p.pool_w = h->pool_hbm;
+    p.n_pool_blocks = g.hbm_cap;
+    p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.out_f32 = out_f32;
+    p.part_o = h->part_o; p.part_ml = h->part_ml; p.tickets = h->tickets;
+    p.finalize = 1;
+    p.n_layers = nl; p.layer0 = l0; p.phys_layers = g.phys_layers;
+    p.lens = h->lens_dev; p.lens_out = h->lens_dev;
+    p.lens_layer_stride = g.max_seqs;
+    p.lens_copy_stride = g.layers * g.max_seqs;
+    for (int l = 0; l < g.layers; ++l)
+        if (h->lens_cur[l]) p.lens_cur_mask |= 1ull << l;
+    p.pool_layer_stride = (uint64_t)g.hbm_cap * g.block_bytes;
+    if (h->lost_copies > 0) {
+        --h->lost_copies;
+        p.drop_first_copy = 1;
+    }
+    long long nu = 0;   // KV blocks in the flat work list (host lengths already include this step's token)
+    for (int l = l0; l < l0 + nl; ++l)
+        for (int s = 0; s < n_seqs; ++s)
+            nu += (long long)std::max(1, (h->bm.length(l, s) + g.BT - 1) / g.BT) * Hg;
+    const int cap = g.max_ctas > 0 ? std::min(g.max_ctas, h->sm_count) : h->sm_count;
+    const int grid = (int)std::max<long long>(1, std::min<long long>(cap, (nu + nw - 1) / nw));
+    CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_RESIDENT, grid, h->stages_res, smem, h->s_compute));
+    ++h->launches;
+    for (int l = l0; l < l0 + nl; ++l) h->lens_cur[l] ^= 1;   // the kernel wrote the advanced lengths to the other copies
+    h->last_fused_layer = -1;
+    return ISV_OK;
+}
+
 int isv_decode_step(isv_kv *h, const void *q, const void *k, const void *v, void *out, float *out_f32,
                     int32_t n_seqs) {
     int rc = check_handle(h, 0, true);
@@ -973,6 +1055,11 @@ int isv_decode_step(isv_kv *h, const void *q, const void *k, const void *v, void
     if (n_seqs < 0 || n_seqs > g.max_seqs) return fail(ISV_EINVAL, "n_seqs %d outside [0, %d]", n_seqs, g.max_seqs);
     const size_t rows = (size_t)n_seqs * g.Hq * g.D;
     const size_t qs = rows * 2, ks = (size_t)n_seqs * g.Hkv * g.D * 2;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(out_f32))
+        return fail(ISV_EINVAL, "q, k, v, out and out_f32 must be 16-byte aligned");
+    size_t smem = 0;
+    if (can_fuse_layers(h, g.layers, n_seqs, &smem))   // the whole step is handed over at once: one launch
+        return decode_layers_fused(h, 0, g.layers, q, k, v, out, out_f32, n_seqs, smem);
     for (int l = 0; l < g.layers; ++l) {
         if ((rc = isv_decode_layer(h, l, (const uint8_t *)q + l * qs, (const uint8_t *)k + l * ks,
                                    (const uint8_t *)v + l * ks, out ? (uint8_t *)out + l * qs : nullptr,
@@ -1033,9 +1120,16 @@ int isv_decode_step_host(isv_kv *h, const void *q, const void *k, const void *v,
     for (int gi = 0; gi < n_groups; ++gi) {
         const int l0 = first[gi], nl = first[gi + 1] - l0;
         CU(cudaStreamWaitEvent(h->s_compute, h->ev_step_in[gi], 0));
-        for (int l = l0; l < l0 + nl; ++l)
-            if ((rc = isv_decode_layer(h, l, dq + l * ql, dk + l * kl, dv + l * kl, dout + l * ql, nullptr, n_seqs)))
+        size_t smem = 0;
+        if (can_fuse_layers(h, nl, n_seqs, &smem)) {   // a group whose inputs have arrived runs as one launch
+            if ((rc = decode_layers_fused(h, l0, nl, dq + l0 * ql, dk + l0 * kl, dv + l0 * kl, dout + l0 * ql, nullptr,
+                                          n_seqs, smem)))
                 return rc;
+        } else {
+            for (int l = l0; l < l0 + nl; ++l)
+                if ((rc = isv_decode_layer(h, l, dq + l * ql, dk + l * kl, dv + l * kl, dout + l * ql, nullptr, n_seqs)))
+                    return rc;
+        }
         CU(cudaEventRecord(h->ev_step_out[gi], h->s_compute));
         CU(cudaStreamWaitEvent(h->s_d2h, h->ev_step_out[gi], 0));
         CU(cudaMemcpyAsync((uint8_t *)out + l0 * ql, dout + l0 * ql, nl * ql, cudaMemcpyDeviceToHost, h->s_d2h));

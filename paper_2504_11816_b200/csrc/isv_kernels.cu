@@ -956,8 +956,12 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     uint8_t *after_data = smem + (size_t)NW * stages * TILE;
     uint64_t *bars = reinterpret_cast<uint64_t *>(after_data) + warp * stages;
     int32_t *meta = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * 8) + warp * stages * V_WORDS;
-    int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * (8 + 4 * V_WORDS));   // [n_seqs + 1]
-    int32_t *slen = ubase + p.n_seqs + 1;   // [n_seqs] tokens to attend (resident mode)
+    // A launch covers NL layers of NSEQ sequences; (layer, sequence) pairs are numbered l * NSEQ + s and are
+    // what "sequence" means below wherever q, out, the new rows, tickets or the work list are indexed.
+    const int NL = (MODE == MODE_RESIDENT && p.n_layers > 1) ? p.n_layers : 1;
+    const int NSEQ = p.n_seqs, NV = NL * NSEQ;
+    int32_t *ubase = reinterpret_cast<int32_t *>(after_data + (size_t)NW * stages * (8 + 4 * V_WORDS));   // [NV + 1]
+    int32_t *slen = ubase + NV + 1;   // [NV] tokens to attend (resident mode)
 
     // Programmatic dependent launch.  This kernel may start while its predecessor in the stream is
     // still running; griddepcontrol.wait returns once that predecessor has completed and its writes
@@ -988,9 +992,16 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     long long NU;
     if (MODE == MODE_RESIDENT) {
         const int len_cap = p.max_blocks * BT;
-        for (int s = threadIdx.x; s < p.n_seqs; s += blockDim.x) {
+        for (int s = threadIdx.x; s < NV; s += blockDim.x) {
             // a length the table row does not cover is never followed into the table
-            const int raw = p.lens[s];
+            int raw;
+            if (NL > 1) {
+                const int l = s / NSEQ, la = p.layer0 + l;
+                raw = p.lens[(size_t)((p.lens_cur_mask >> la) & 1) * p.lens_copy_stride +
+                             (size_t)la * p.lens_layer_stride + (s - l * NSEQ)];
+            } else {
+                raw = p.lens[s];
+            }
             const int len = min(max(raw, 0) + fused, len_cap);
             if (len != raw + fused) atomicOr(p.status, ISV_STATUS_BAD_LENGTH);
             slen[s] = len;
@@ -1000,20 +1011,20 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         __syncthreads();
         if (warp == 0) {
             int carry = 0;
-            for (int base = 0; base < p.n_seqs; base += 32) {
+            for (int base = 0; base < NV; base += 32) {
                 const int i = base + lane;
-                int v = i < p.n_seqs ? ubase[i + 1] : 0;
+                int v = i < NV ? ubase[i + 1] : 0;
 #pragma unroll
                 for (int d = 1; d < 32; d <<= 1) {
                     const int t = __shfl_up_sync(kFull, v, d);
                     if (lane >= d) v += t;
                 }
-                if (i < p.n_seqs) ubase[i + 1] = carry + v;
+                if (i < NV) ubase[i + 1] = carry + v;
                 carry += __shfl_sync(kFull, v, 31);
             }
         }
         __syncthreads();
-        NU = ubase[p.n_seqs];
+        NU = ubase[NV];
     } else {
         NU = (long long)p.cu_count * Hg;
     }
@@ -1034,6 +1045,8 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
 
     // ---- producer state (identical in all lanes except the two per-entry values)
     int pu_s = 0, pu_hg = 0, pu_nc = 1, pu_wf = 0, pu_wfslot = 0;
+    int pu_row = 0;                                // table row (sequence within the layer) of the open segment
+    const uint8_t *pu_pool = p.pool, *pu_tail = p.tail;   // its layer's slabs
     bool pu_first = true, range_first = true;   // the open segment is / the next one will be the first of its range
     bool seg_start = false;                     // the next visit is the first of its segment
     int pu_len = 0, pu_jlast = -1, pu_j0 = 0, pu_n = 0;   // entries of the open unit: [pu_j0, pu_j0 + pu_n)
@@ -1047,7 +1060,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     int prod_vis = 0, inflight = 0;     // ring position of the next visit to emit; visits emitted and not consumed
     bool drop_copy = p.drop_first_copy && blockIdx.x == 0 && warp == 0;   // failure injection, see DecodeParams
     if (MODE == MODE_RESIDENT) {   // sequence of the first unit: largest s with ubase[s] <= u_next
-        int lo = 0, hi = p.n_seqs - 1;
+        int lo = 0, hi = NV - 1;
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
             if (ubase[mid] <= u_next) lo = mid; else hi = mid - 1;
@@ -1087,15 +1100,15 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
                     if (j < pu_j0 + pu_n) {
                         int32_t e;
                         if (MODE == MODE_RESIDENT) {
-                            e = p.table[(size_t)pu_s * p.table_stride + j];
+                            e = p.table[(size_t)pu_row * p.table_stride + j];
                             if (e != ISV_BLOCK_NONE) {
                                 if (e & ISV_BLOCK_HOST_BIT) {   // only the newest block of a sequence is read from its tail slot
-                                    valid = (j == pu_jlast) && (p.tail != nullptr);
-                                    src = p.tail + (uint64_t)pu_s * block_bytes;
+                                    valid = (j == pu_jlast) && (pu_tail != nullptr);
+                                    src = pu_tail + (uint64_t)pu_row * block_bytes;
                                 } else {
                                     valid = e >= 0 && e < p.n_pool_blocks;
                                     if (!valid) atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
-                                    src = p.pool + (uint64_t)e * block_bytes;
+                                    src = pu_pool + (uint64_t)e * block_bytes;
                                 }
                             }
                             if (j == pu_jlast) nt = (pu_len - j * BT - fused) | (fused ? 256 : 0);
@@ -1125,6 +1138,14 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             if (MODE == MODE_RESIDENT) {
                 const int x = u_next;
                 while (x >= ubase[pu_s + 1]) ++pu_s;
+                pu_row = pu_s;
+                if (NL > 1) {
+                    const int l = pu_s / NSEQ;
+                    const int slab = (p.layer0 + l) % p.phys_layers;
+                    pu_row = pu_s - l * NSEQ;
+                    pu_pool = p.pool + (uint64_t)slab * p.pool_layer_stride;
+                    pu_tail = p.tail ? p.tail + (uint64_t)slab * p.tail_layer_stride : nullptr;
+                }
                 pu_len = slen[pu_s];
                 const int nblk = (pu_len + BT - 1) / BT;
                 const int nb = max(1, nblk);
@@ -1214,23 +1235,39 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     // (pool, or the sequence's tail slot when that block is host-flagged).  Nothing in this launch
     // reads those slots: the new token is attended to from k_new / v_new directly.
     if (fused) {
-        const int rows = p.n_seqs * 2 * p.Hkv;
+        const int rows = NV * 2 * p.Hkv;
         const int row_vecs = D * 2 / 16;
         for (int r = blockIdx.x * NW + warp; r < rows; r += gridDim.x * NW) {
             const int s = r / (2 * p.Hkv);
             const int kv = (r / p.Hkv) & 1, h = r % p.Hkv;
             const int len = slen[s] - 1;   // length before this step's token
             const int j = len / BT, slot = len % BT;
-            const int32_t e = p.table[(size_t)s * p.table_stride + j];
+            int row = s;                   // table row; the layer's slabs and length copy to write
+            uint8_t *pool_w = p.pool_w, *tail_w = p.tail_w;
+            int32_t *lens_out = p.lens_out;
+            bool store = true;
+            if (NL > 1) {
+                const int l = s / NSEQ, la = p.layer0 + l;
+                const int slab = la % p.phys_layers;
+                row = s - l * NSEQ;
+                pool_w += (uint64_t)slab * p.pool_layer_stride;
+                if (tail_w) tail_w += (uint64_t)slab * p.tail_layer_stride;
+                lens_out = p.lens_out + (size_t)(((p.lens_cur_mask >> la) & 1) ^ 1) * p.lens_copy_stride +
+                           (size_t)la * p.lens_layer_stride;
+                store = l + p.phys_layers >= NL;   // a later layer of this launch writes the same slot
+            }
+            const int32_t e = p.table[(size_t)row * p.table_stride + j];
             uint8_t *base = nullptr;
             if (e != ISV_BLOCK_NONE) {
                 if (e & ISV_BLOCK_HOST_BIT) {
-                    if (p.tail_w) base = p.tail_w + (uint64_t)s * block_bytes;
+                    if (tail_w) base = tail_w + (uint64_t)row * block_bytes;
                 } else if (e >= 0 && e < p.n_pool_blocks) {
-                    base = p.pool_w + (uint64_t)e * block_bytes;
+                    base = pool_w + (uint64_t)e * block_bytes;
                 }
             }
-            if (base) {
+            if (base && !store) {
+                // nothing to write
+            } else if (base) {
                 if (lane < row_vecs) {
                     const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v_new : p.k_new) +
                                          ((size_t)s * p.Hkv + h) * (D * 2) + lane * 16;
@@ -1241,7 +1278,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             } else if (lane == 0) {
                 atomicOr(p.status, ISV_STATUS_BAD_BLOCK_ID);
             }
-            if (kv == 0 && h == 0 && lane == 0) p.lens_out[s] = len + 1;
+            if (kv == 0 && h == 0 && lane == 0) lens_out[row] = len + 1;
         }
     }
 

@@ -45,6 +45,22 @@ struct DecodeParams {
     const void *k_new, *v_new;  // [n_seqs][Hkv][D] 16-bit, or NULL
     int32_t *lens_out;          // [n_seqs]
     uint8_t *pool_w, *tail_w;   // writable aliases of pool / tail
+    // several layers in one launch (resident mode with fused append only): n_layers > 1 makes the launch
+    // cover logical layers layer0 .. layer0 + n_layers - 1 of one decode step.  The work list is then the
+    // flat space of KV blocks ordered by (layer, sequence, head group, block), cut evenly over the grid's
+    // warps as before, so the start-up and the tail of a launch are paid once per step instead of once per
+    // layer.  q, k_new, v_new, out and out_f32 hold the layers back to back ([layer][n_seqs][heads][D]), so a
+    // (layer, sequence) pair indexes them like a sequence number layer * n_seqs + s; `pool` / `tail` point at
+    // physical slab 0 and layer l uses slab l % phys_layers; `lens` points at the first of two copies of
+    // [layers][lens_layer_stride] lengths, bit l of lens_cur_mask says which copy is current for layer l, and
+    // the advanced lengths go to the other one.  Where several layers of the launch share a slab only the
+    // last of them stores its token (the earlier rows would be overwritten anyway; nothing in the launch
+    // reads them).
+    int32_t n_layers;           // 0 or 1: one layer, the fields below are unused
+    int32_t layer0, phys_layers;
+    int32_t lens_layer_stride, lens_copy_stride;   // in elements
+    uint64_t lens_cur_mask;
+    uint64_t pool_layer_stride, tail_layer_stride; // bytes between physical slabs
     // inputs / outputs
     const void *q;              // [n_seqs][Hq][D] 16-bit
     void *out;                  // [n_seqs][Hq][D] 16-bit or NULL
@@ -144,7 +160,7 @@ int decode_default_stages(int D, int BT, int GT);
 
 // Bytes of dynamic shared memory the decode kernel needs for `stages` ring
 // stages (one K or V tile each) per warp.
-size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode);
+size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode);   // max_seqs: sequences x layers of a launch
 
 // Launchers return the CUDA error of the launch.
 cudaError_t decode_configure(int D, int GT, int BT, bool bf16, int mode, size_t smem);

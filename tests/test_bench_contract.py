@@ -66,7 +66,7 @@ def test_cuda_arm_prints_one_json_line_with_roofline_and_clocks():
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["peak"] > 0
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
-    assert d["gpu_launches"] >= 4 * 2 and d["value"] > 0 and d["n_gpus"] == 1
+    assert d["gpu_launches"] >= 4 and d["value"] > 0 and d["n_gpus"] == 1      # a launch per step (all layers)
     assert d["e2e"]["value"] > 0 and d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > 0
     assert d["cpu_baseline"]["value"] > 0 and d["cpu_baseline"]["kind"] == "oracle"
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}

@@ -344,12 +344,17 @@ def test_link_probe_reports_plausible_rates():
 # ---------------------------------------------------------------- launch chains, bad lengths, failure paths
 
 @pytest.mark.parametrize("layers,phys,ctas,f", [(2, 2, 4, 0.0), (3, 3, 8, 0.0), (3, 2, 6, 0.0), (2, 2, 5, 0.5)])
-def test_steps_enqueued_back_to_back_on_small_grids(layers, phys, ctas, f):
+@pytest.mark.parametrize("per_layer", [True, False])
+def test_steps_enqueued_back_to_back_on_small_grids(layers, phys, ctas, f, per_layer, monkeypatch):
     """Several whole steps are enqueued without a host wait in between, on grids far below the SM count.
     Launches then follow one another as fast as programmatic dependent launch allows, and a layer's launch of
     step t+1 must still see the lengths and the K/V rows its launch of step t wrote (with two layers the
     writer is only two launches back; with shared slabs likewise).  Every step's output is compared with
     the reference afterwards, and the cache is read back bit for bit."""
+    if per_layer:      # one launch per layer even where a whole step could be one launch
+        monkeypatch.setenv("ISV_LAYERS_PER_LAUNCH", "1")
+    elif f > 0:
+        pytest.skip("with offloaded blocks a step is always one launch per layer")
     steps = 7
     w = small(batch=8, steps=steps, f=f, perm=13, ctx=(1900, 2040), layers=layers, q_heads=4, kv_heads=4,
               head_dim=128, seed=23)
@@ -383,6 +388,52 @@ def test_steps_enqueued_back_to_back_on_small_grids(layers, phys, ctas, f):
             hz.check_step(res)
         assert np.array_equal(B.isv_seq_lens_host(hz.h, layers - 1, w.batch), hz.cur)
         hz.check_gather(layers=range(layers - phys, layers))
+
+
+@pytest.mark.parametrize("q_heads,kv_heads,head_dim,dtype", [(4, 4, 128, "f16"), (8, 2, 128, "bf16"), (6, 6, 80, "f16"),
+                                                             (16, 2, 64, "f16")])
+@pytest.mark.parametrize("layers,phys,ctas", [(5, 5, 0), (5, 2, 3), (4, 4, 1)])
+def test_whole_step_as_one_launch(q_heads, kv_heads, head_dim, dtype, layers, phys, ctas):
+    """With nothing offloaded isv_decode_step runs all layers' append + attention as one launch whose work list
+    spans the layers.  Ragged lengths (an empty sequence, one token, block boundaries), layers that share
+    slabs, and grids of 1, 3 and all CTAs; every output row against the reference, lengths and cache read back."""
+    lens = [0, 1, 15, 16, 17, 100, 257, 330]
+    steps = 18                                    # crosses a block boundary for every sequence
+    w = small(batch=len(lens), steps=steps + 1, f=0.0, perm=17, ctx=(0, 330), layers=layers, q_heads=q_heads,
+              kv_heads=kv_heads, head_dim=head_dim, dtype=dtype, seed=29)
+    td = W.torch_dtype(w.dtype)
+    with Harness(w, lens=lens, max_ctas=ctas, phys_layers=phys) as hz:
+        hz.fill()
+        launches0 = B.isv_kv_info(hz.h).kernel_launches
+        updates = 0
+        for t in range(steps):
+            ks, vs, qs = zip(*[W.host_step(w, hz.rng) for _ in range(layers)])
+            k, v, q = (np.stack(x) for x in (ks, vs, qs))
+            kd, vd, qd = (bits_to_dev(x, w.dtype) for x in (k, v, q))
+            of = torch.full((layers, w.batch, w.q_heads, w.head_dim), float("nan"), device="cuda")
+            o16 = torch.zeros((layers, w.batch, w.q_heads, w.head_dim), device="cuda", dtype=td)
+            torch.cuda.synchronize()
+            updates += int(np.any(hz.cur % 16 == 0))          # a step that opens new blocks also updates the table
+            B.isv_decode_step(hz.h, qd, kd, vd, o16, of, w.batch)
+            assert B.isv_sync(hz.h) == 0
+            res = []
+            for layer in range(layers):
+                if phys < layers:
+                    hz.shadow.store_at(layer % phys, k[layer], v[layer], hz.cur.tolist())
+                    ref = hz.reference(layer, q[layer], lens=hz.cur + 1)
+                else:
+                    hz.shadow.append(layer, k[layer], v[layer])
+                    ref = None
+                res.append((q[layer], of[layer].cpu().numpy(), dev_to_bits(o16[layer]), ref))
+            hz.cur += 1
+            hz.check_step(res)
+        # one attention launch per step, whatever the number of layers
+        assert B.isv_kv_info(hz.h).kernel_launches - launches0 == steps + updates
+        for layer in range(layers):
+            assert np.array_equal(B.isv_seq_lens_host(hz.h, layer, w.batch), hz.cur)
+        hz.check_gather(layers=range(layers - phys, layers))
+        # the per-layer calls continue from the same state
+        hz.check_step(hz.step(fused=True))
 
 
 def test_device_lengths_beyond_the_table_row_are_clamped_and_flagged():
