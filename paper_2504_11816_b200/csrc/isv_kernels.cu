@@ -54,7 +54,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: false when the phase did not complete within `limit` polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit) {
-    for (uint32_t i = 0; i < limit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;   // the usual case: the copy landed while the warp computed
+    for (uint32_t i = 1; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 256) __nanosleep(64);
     }
@@ -104,6 +105,15 @@ __device__ __forceinline__ void ffma2(float &d0, float &d1, float a0, float a1, 
     d0 = fmaf(a0, b0, d0);
     d1 = fmaf(a1, b1, d1);
 #endif
+}
+
+// 2^x by the special-function unit alone (ex2.approx: relative error about 2^-22, 2^0 = 1 exactly, results
+// below the normal range flush to zero).  exp2f adds a range-scaling sequence around the same instruction;
+// softmax weights need neither the extra bits nor denormal results, and the tile loops run it per token.
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 template <bool BF16>
@@ -187,28 +197,31 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
         cvt8<BF16>(reinterpret_cast<const uint4 *>(sK + tt * ROW)[NVF * 8 + (sub & 1)], kf);
 #pragma unroll
         for (int g = 0; g < GT; ++g) {
-            float tp = 0.f;
+            float tp = 0.f, tp1 = 0.f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) tp = fmaf(q[g][NVF * 8 + e], kf[e], tp);
+            for (int e = 0; e < 8; e += 2) ffma2(tp, tp1, q[g][NVF * 8 + e], q[g][NVF * 8 + e + 1], kf[e], kf[e + 1]);
+            tp += tp1;
             tp += __shfl_xor_sync(kFull, tp, 1);   // lanes 2i and 2i+1 of a group: the two tail chunks of one token
 #pragma unroll
             for (int i = 0; i < NQ; ++i)   // the tail of this group's token of pass i was taken by group (grp - i) mod 4
                 sc[i][g] += __shfl_sync(kFull, tp, ((grp - i) & 3) * 8 + 2 * i);
         }
     }
+    if (ntok < BT) {   // slots past the sequence end hold unspecified bits: their scores are replaced
 #pragma unroll
-    for (int i = 0; i < NQ; ++i)   // slots past the sequence end hold unspecified bits: their scores are replaced
-        if (4 * i + grp >= ntok) {
+        for (int i = 0; i < NQ; ++i)
+            if (4 * i + grp >= ntok) {
 #pragma unroll
-            for (int g = 0; g < GT; ++g) sc[i][g] = kNegBig;
-        }
+                for (int g = 0; g < GT; ++g) sc[i][g] = kNegBig;
+            }
+    }
 #pragma unroll
     for (int g = 0; g < GT; ++g) {
         float mx = sc[0][g];
 #pragma unroll
         for (int i = 1; i < NQ; ++i) mx = fmaxf(mx, sc[i][g]);
         if (mx > m[g]) {
-            const float r = exp2f(m[g] - mx);
+            const float r = fast_exp2(m[g] - mx);
             l[g] *= r;
 #pragma unroll
             for (int e = 0; e < NV * 8; ++e) o[g][e] *= r;
@@ -232,7 +245,7 @@ __device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp
         if (t < ntok) {   // slots past the sequence end hold unspecified bits: never touch them
 #pragma unroll
             for (int g = 0; g < GT; ++g) {
-                pwv[i][g] = exp2f(sc[i][g] - m[g]);
+                pwv[i][g] = fast_exp2(sc[i][g] - m[g]);
                 l[g] += pwv[i][g];
             }
             const uint4 *vrow = reinterpret_cast<const uint4 *>(sV + t * ROW);
@@ -554,7 +567,7 @@ struct MmaMath {
 
     // Raises the running maxima to (n0, n1) and rescales l and the accumulators accordingly.
     __device__ __forceinline__ void raise_max(float n0, float n1) {
-        const float r0 = exp2f(m[0] - n0), r1 = exp2f(m[1] - n1);
+        const float r0 = fast_exp2(m[0] - n0), r1 = fast_exp2(m[1] - n1);
         l[0] *= r0;
         l[1] *= r1;
 #pragma unroll
@@ -599,8 +612,8 @@ struct MmaMath {
         if (__any_sync(kFull, mx0 > m[0] || mx1 > m[1])) raise_max(fmaxf(m[0], mx0), fmaxf(m[1], mx1));
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            x[i] = exp2f(x[i] - m[0]);
-            y[i] = exp2f(y[i] - m[1]);
+            x[i] = fast_exp2(x[i] - m[0]);
+            y[i] = fast_exp2(y[i] - m[1]);
         }
         l[0] += (x[0] + x[1]) + (x[2] + x[3]);
         l[1] += (y[0] + y[1]) + (y[2] + y[3]);
@@ -1189,11 +1202,13 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         if (lane == 0) {
             int32_t *mt = meta + prod_vis * V_WORDS;
             mt[V_INFO] = ntok | flags;
-            mt[V_SEQ] = pu_s;
-            mt[V_HG] = pu_hg;
-            mt[V_NC] = pu_nc;
-            mt[V_WF] = pu_wf;
-            mt[V_PACK] = pu_wfslot | (pu_first ? 2 : 0) | (cur_range << 2);   // three fields in one word
+            if (flags & (VF_FIRST | VF_LAST)) {   // the consumer reads these at segment boundaries only
+                mt[V_SEQ] = pu_s;
+                mt[V_HG] = pu_hg;
+                mt[V_NC] = pu_nc;
+                mt[V_WF] = pu_wf;
+                mt[V_PACK] = pu_wfslot | (pu_first ? 2 : 0) | (cur_range << 2);   // three fields in one word
+            }
             const uint32_t bar = smem_u32(&bars[2 * prod_vis]);
             if (ksrc) {
                 mbar_arrive_expect_tx(bar, TILE);
