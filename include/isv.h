@@ -235,11 +235,14 @@ int isv_set_zero_copy(isv_kv *h, int32_t on);
 /* One decode step of all layers: the result of isv_decode_layer for l in 0..layers-1.
  * Device arrays: q, out (16-bit) and out_f32 (fp32) [layers][n_seqs][q_heads][head_dim];
  * k, v [layers][n_seqs][kv_heads][head_dim].  out_dev and out_f32_dev may each be NULL, not both.
- * Because all layers' inputs are handed over at once, a cache with offload_frac = 0 is served by ONE
- * launch whose work list spans the layers (the start-up and the tail of a launch are then paid once per
- * step, which matters when a layer's KV is read in under 100 microseconds); with offloaded blocks, or
- * with per-layer timing on, it is one launch per layer as in isv_decode_layer.  A caller whose layers
- * depend on one another (a real model) uses isv_decode_layer per layer. */
+ * Because all layers' inputs are handed over at once, the resident attention (and the appends) of up to
+ * phys_layers consecutive layers run as ONE launch whose work list spans those layers: the start-up and
+ * the tail of a launch are then paid once per step instead of once per layer, which matters when a
+ * layer's KV is read in under 100 microseconds.  With offloaded blocks each layer's staged launches and
+ * merge follow that launch, and the copy engine's queue is filled for all of them at once.  (Layers that
+ * share a physical slab are never put into one launch.  With offload_frac = 0 and per-layer timing on it
+ * is one launch per layer.)  A caller whose layers depend on one another (a real model) uses
+ * isv_decode_layer per layer. */
 int isv_decode_step(isv_kv *h, const void *q_dev, const void *k_dev, const void *v_dev,
                     void *out_dev, float *out_f32_dev, int32_t n_seqs);
 

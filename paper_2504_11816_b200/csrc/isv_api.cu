@@ -105,6 +105,7 @@ struct isv_kv {
     int stages_res = 0, stages_stg = 0;
     size_t smem_res = 0, smem_stg = 0;
     int smem_limit = 0;                    // opt-in shared memory per block of the device
+    int res_layers = 1;                    // layers the resident-result and running-state buffers hold
     uint64_t launches = 0;                 // kernels launched so far
     int last_fused_layer = -1;             // layer of the latest fused decode launch if nothing else of ours
                                            // was launched on the compute stream since, else -1
@@ -344,6 +345,14 @@ int upload_plan(isv_kv *h, const OffPlan &pl, PlanSlot **out) {
     return ISV_OK;
 }
 
+// One layer of a step whose resident part has already been enqueued for all layers by a single launch:
+// where that launch left the layer's unnormalised result, the layer's own running state of the offloaded
+// part, and how many CTAs a staged launch may take (the resident launch leaves that many SMs free).
+struct FusedLayer {
+    float *res_o, *res_ml, *run_o, *run_ml;
+    int staged_grid_cap;
+};
+
 struct AppendPlan {
     std::vector<TableUpdate> upd;   // table entries of blocks allocated for this step
     std::vector<int> flush;         // sequences whose host-flagged newest block becomes full
@@ -478,10 +487,17 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
     if ((rc = dev_alloc((void **)&h->tickets, tickets_bytes(g), &h->scratch_bytes, "tickets"))) return bail(rc);
     CUB(cudaMemset(h->tickets, 0, tickets_bytes(g)));
     if (g.host_cap > 0) {
-        if ((rc = dev_alloc((void **)&h->res_o, rows * g.D * 4, &h->scratch_bytes, "resident result"))) return bail(rc);
-        if ((rc = dev_alloc((void **)&h->res_ml, rows * 2 * 4, &h->scratch_bytes, "resident result"))) return bail(rc);
-        if ((rc = dev_alloc((void **)&h->run_o, rows * g.D * 4, &h->scratch_bytes, "running state"))) return bail(rc);
-        if ((rc = dev_alloc((void **)&h->run_ml, rows * 2 * 4, &h->scratch_bytes, "running state"))) return bail(rc);
+        // one copy per layer of a launch where the resident part of several layers can be a single launch (its
+        // per-layer results then wait for the layers' offloaded parts), else one; a launch covers at most
+        // phys_layers layers
+        if (g.phys_layers > 1 && g.layers <= 64 &&
+            decode_smem_bytes(g.D, g.BT, g.GT, h->stages_res, 2 * g.max_seqs, MODE_RESIDENT) <= (size_t)smem_limit)
+            h->res_layers = g.phys_layers;
+        const size_t nl = (size_t)h->res_layers;
+        if ((rc = dev_alloc((void **)&h->res_o, nl * rows * g.D * 4, &h->scratch_bytes, "resident result"))) return bail(rc);
+        if ((rc = dev_alloc((void **)&h->res_ml, nl * rows * 2 * 4, &h->scratch_bytes, "resident result"))) return bail(rc);
+        if ((rc = dev_alloc((void **)&h->run_o, nl * rows * g.D * 4, &h->scratch_bytes, "running state"))) return bail(rc);
+        if ((rc = dev_alloc((void **)&h->run_ml, nl * rows * 2 * 4, &h->scratch_bytes, "running state"))) return bail(rc);
     }
     // events
     h->ev_ready.resize(g.ring);
@@ -782,7 +798,7 @@ int isv_kv_append(isv_kv *h, int32_t layer, const void *k, const void *v, int32_
 // (the device lengths then still hold the values before the append and the kernel advances them).
 static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float *out_f32,
                        const int32_t *block_table_dev, const int32_t *seq_lens_dev, int32_t n_seqs,
-                       const void *k_new, const void *v_new, bool tables_settled) {
+                       const void *k_new, const void *v_new, bool tables_settled, const FusedLayer *fc = nullptr) {
     int rc = ISV_OK;
     const Geometry &g = h->g;
     if (n_seqs < 0 || n_seqs > g.max_seqs) return fail(ISV_EINVAL, "n_seqs %d outside [0, %d]", n_seqs, g.max_seqs);
@@ -806,8 +822,9 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
         le->bytes_off = pl.bytes_offloaded;
         le->bytes_staged = (offloaded && !h->zero_copy) ? pl.bytes_staged : 0;
         le->n_chunks = (int)pl.chunks.size();
-        CU(cudaEventRecord(le->d0, h->s_compute));
+        if (!fc) CU(cudaEventRecord(le->d0, h->s_compute));   // (a step-wide resident launch recorded it already)
     }
+    float *run_o = fc ? fc->run_o : h->run_o, *run_ml = fc ? fc->run_ml : h->run_ml;
 
     DecodeParams base{};
     base.table = block_table_dev ? block_table_dev : h->table_dev;
@@ -824,10 +841,12 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
     if (offloaded) {
         // ---- staging engine: host blocks stream through the ring while the resident kernel runs
         PlanSlot *ps = nullptr;
-        CU(cudaEventRecord(h->ev_q, h->s_compute));          // q (and everything before) is ready
-        CU(cudaStreamWaitEvent(h->s_off, h->ev_q, 0));
+        if (!fc) {   // (with a step-wide resident launch the offload stream was released before that launch)
+            CU(cudaEventRecord(h->ev_q, h->s_compute));          // q (and everything before) is ready
+            CU(cudaStreamWaitEvent(h->s_off, h->ev_q, 0));
+        }
         if ((rc = upload_plan(h, pl, &ps))) return rc;
-        CU(cudaMemsetAsync(h->run_ml, 0, (size_t)n_seqs * g.Hq * 2 * 4, h->s_off));
+        CU(cudaMemsetAsync(run_ml, 0, (size_t)n_seqs * g.Hq * 2 * 4, h->s_off));
         if (h->flush_recorded[phys]) CU(cudaStreamWaitEvent(h->zero_copy ? h->s_off : h->s_copy, h->ev_flush[phys], 0));
         if (le) {
             CU(cudaEventRecord(le->c0, h->s_copy));
@@ -863,11 +882,11 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
             p.cblk = ps->dev + ps->off_blk;
             p.cu_first = ch.unit_begin;
             p.cu_count = ch.unit_end - ch.unit_begin;
-            p.acc_o = h->run_o;
-            p.acc_ml = h->run_ml;
+            p.acc_o = run_o;
+            p.acc_ml = run_ml;
             const long long nu2 = (long long)p.cu_count * Hg;
             // reading in place needs few CTAs to saturate the link and leaves the other SMs to the resident kernel
-            const long long cap2 = h->zero_copy ? std::max(1, h->sm_count / 4) : h->sm_count;
+            const long long cap2 = h->zero_copy ? std::max(1, h->sm_count / 4) : (fc ? fc->staged_grid_cap : h->sm_count);
             const int grid = (int)std::max<long long>(1, std::min<long long>(cap2, (nu2 + nw - 1) / nw));
             CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_STAGED, grid, h->stages_stg, h->smem_stg, h->s_off));
             ++h->launches;
@@ -886,7 +905,7 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
     }
 
     // ---- resident part
-    {
+    if (!fc) {
         DecodeParams p = base;
         p.pool = h->pool_hbm + slab_hbm(h, layer);
         p.tail = h->tail ? h->tail + slab_tail(h, layer) : nullptr;
@@ -924,10 +943,12 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
         h->last_fused_layer = k_new ? layer : -1;
     }
 
-    if (offloaded) {
-        CU(cudaStreamWaitEvent(h->s_compute, h->ev_off_done, 0));
+    if (offloaded || fc) {
+        if (offloaded) CU(cudaStreamWaitEvent(h->s_compute, h->ev_off_done, 0));
+        else CU(cudaMemsetAsync(run_ml, 0, (size_t)n_seqs * g.Hq * 2 * 4, h->s_compute));   // nothing offloaded here: an empty running state
         MergeParams mp{};
-        mp.res_o = h->res_o; mp.res_ml = h->res_ml; mp.run_o = h->run_o; mp.run_ml = h->run_ml;
+        mp.res_o = fc ? fc->res_o : h->res_o; mp.res_ml = fc ? fc->res_ml : h->res_ml;
+        mp.run_o = run_o; mp.run_ml = run_ml;
         mp.out = out; mp.out_f32 = out_f32;
         mp.rows = n_seqs * g.Hq; mp.D = g.D; mp.bf16 = bf16 ? 1 : 0;
         if (le) CU(cudaEventRecord(le->m0, h->s_compute));
@@ -969,41 +990,79 @@ int isv_decode_layer(isv_kv *h, int32_t layer, const void *q, const void *k, con
     return flush_tails(h, layer, ap.flush);
 }
 
-// Whether layers [l0, l0 + nl) of a step can run as one launch: nothing of the cache is offloaded (no
-// staging, no tail slots, no per-layer merge), per-layer timing is off (there is no per-layer launch to
-// time), and the kernel's per-(layer, sequence) tables fit in shared memory beside the full ring.
-static bool can_fuse_layers(const isv_kv *h, int nl, int n_seqs, size_t *smem) {
+// How many of the layers l0, l0 + 1, ... (at most nl) can have their resident attention (and appends) in one
+// launch; 1 = none beyond the first, i.e. the per-layer path.  A launch never covers two layers that share a
+// physical slab, so at most phys_layers layers: layers sharing a slab then keep the order of separate
+// launches (the later one's token stays), and a benchmark that holds fewer slabs than layers cannot have two
+// layers of a launch stream the same bytes at the same time and find them in L2.  With nothing offloaded
+// per-layer timing must be off (there is no per-layer launch to time); with part of the cache on the host
+// the blocks must be staged through the ring and the per-layer result buffers exist.  The kernel's
+// per-(layer, sequence) tables must fit in shared memory beside the full ring.
+static int fusable_layers(const isv_kv *h, int nl, int n_seqs, size_t *smem) {
     const Geometry &g = h->g;
-    if (nl < 2 || n_seqs < 1 || h->timing || g.host_cap != 0 || g.layers > 64) return false;
+    nl = std::min(nl, g.phys_layers);
+    if (nl < 2 || n_seqs < 1 || g.layers > 64) return 1;
     if (const char *e = getenv("ISV_LAYERS_PER_LAUNCH"))   // tuning knob: 1 = one launch per layer
-        if (atoi(e) == 1) return false;
-    const size_t b = decode_smem_bytes(g.D, g.BT, g.GT, h->stages_res, nl * n_seqs, MODE_RESIDENT);
-    if (b > (size_t)h->smem_limit) return false;
-    *smem = b;
-    return true;
+        if (atoi(e) == 1) return 1;
+    if (g.host_cap == 0) {
+        if (h->timing) return 1;
+    } else {
+        if (h->zero_copy || h->res_layers < 2) return 1;
+        nl = std::min(nl, h->res_layers);
+    }
+    while (nl >= 2 && decode_smem_bytes(g.D, g.BT, g.GT, h->stages_res, nl * n_seqs, MODE_RESIDENT) > (size_t)h->smem_limit)
+        --nl;
+    if (nl < 2) return 1;
+    *smem = decode_smem_bytes(g.D, g.BT, g.GT, h->stages_res, nl * n_seqs, MODE_RESIDENT);
+    return nl;
 }
 
-// Layers [l0, l0 + nl) of one decode step (append + attention each) as ONE launch of the resident kernel.
-// q, out, out_f32: [nl][n_seqs][q_heads][head_dim]; k, v: [nl][n_seqs][kv_heads][head_dim], device.
+// Layers [l0, l0 + nl) of one decode step with ONE launch of the resident kernel for all of them (appends
+// fused).  q, out, out_f32: [nl][n_seqs][q_heads][head_dim]; k, v: [nl][n_seqs][kv_heads][head_dim], device.
+// With host-resident blocks the launch leaves every layer's unnormalised result, a few SMs stay free for the
+// staged launches, and the layers' offloaded parts and merges are enqueued behind it: the copy engine's queue
+// is filled for the whole step at once and never waits for a resident launch.
 static int decode_layers_fused(isv_kv *h, int l0, int nl, const void *q, const void *k, const void *v, void *out,
                                float *out_f32, int n_seqs, size_t smem) {
     const Geometry &g = h->g;
     int rc = ISV_OK;
+    const bool split = g.host_cap > 0;
     // host side of the appends; nothing stays changed when a layer cannot take its token
     for (int l = l0; l < l0 + nl; ++l)
         for (int s = 0; s < n_seqs; ++s)
             if (h->bm.length(l, s) >= g.max_tokens)
                 return fail(ISV_ECAPACITY, "sequence %d is full (%d tokens)", s, h->bm.length(l, s));
-    AppendPlan ap;
+    std::vector<AppendPlan> aps(nl);
+    std::vector<TableUpdate> upd;
     for (int l = l0; l < l0 + nl; ++l) {
-        if ((rc = append_bookkeeping(h, l, n_seqs, &ap))) {
+        AppendPlan &ap = aps[l - l0];
+        rc = append_bookkeeping(h, l, n_seqs, &ap);
+        upd.insert(upd.end(), ap.upd.begin(), ap.upd.end());
+        if (rc) {
             for (int lb = l0; lb < l; ++lb)
                 for (int s = 0; s < n_seqs; ++s) --h->bm.length(lb, s);
-            push_updates(h, ap.upd);   // blocks handed out so far stay allocated
+            push_updates(h, upd);   // blocks handed out so far stay allocated
             return rc;
         }
     }
-    if ((rc = push_updates(h, ap.upd))) return rc;
+    if ((rc = push_updates(h, upd))) return rc;
+    if (split)   // a tail slot about to take a new block must have finished its write-back
+        for (int l = l0; l < l0 + nl; ++l) {
+            const int pl = l % g.phys_layers;
+            if (aps[l - l0].new_host_block && h->flush_recorded[pl]) CU(cudaStreamWaitEvent(h->s_compute, h->ev_flush[pl], 0));
+        }
+    if (h->timing) {
+        for (int l = l0; l < l0 + nl; ++l) {
+            h->lev[l].have_append = false;
+            h->lev[l].fused_append = true;
+            h->lev[l].bytes_app = (uint64_t)n_seqs * g.kappa;
+            CU(cudaEventRecord(h->lev[l].d0, h->s_compute));
+        }
+    }
+    if (split) {   // the offload stream may start on the step's staged launches now: they do not depend on the resident launch
+        CU(cudaEventRecord(h->ev_q, h->s_compute));
+        CU(cudaStreamWaitEvent(h->s_off, h->ev_q, 0));
+    }
 
     const bool bf16 = g.dtype == ISV_BF16;
     const int Hg = g.Hkv * g.P;
@@ -1018,10 +1077,12 @@ static int decode_layers_fused(isv_kv *h, int l0, int nl, const void *q, const v
     p.block_bytes = g.block_bytes;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)g.D));
     p.pool = h->pool_hbm; p.pool_w = h->pool_hbm;
+    p.tail = h->tail; p.tail_w = h->tail;
     p.n_pool_blocks = g.hbm_cap;
     p.q = q; p.k_new = k; p.v_new = v; p.out = out; p.out_f32 = out_f32;
     p.part_o = h->part_o; p.part_ml = h->part_ml; p.tickets = h->tickets;
-    p.finalize = 1;
+    p.acc_o = h->res_o; p.acc_ml = h->res_ml;
+    p.finalize = split ? 0 : 1;
     p.n_layers = nl; p.layer0 = l0; p.phys_layers = g.phys_layers;
     p.lens = h->lens_dev; p.lens_out = h->lens_dev;
     p.lens_layer_stride = g.max_seqs;
@@ -1029,6 +1090,7 @@ static int decode_layers_fused(isv_kv *h, int l0, int nl, const void *q, const v
     for (int l = 0; l < g.layers; ++l)
         if (h->lens_cur[l]) p.lens_cur_mask |= 1ull << l;
     p.pool_layer_stride = (uint64_t)g.hbm_cap * g.block_bytes;
+    p.tail_layer_stride = (uint64_t)g.max_seqs * g.block_bytes;
     if (h->lost_copies > 0) {
         --h->lost_copies;
         p.drop_first_copy = 1;
@@ -1037,12 +1099,64 @@ static int decode_layers_fused(isv_kv *h, int l0, int nl, const void *q, const v
     for (int l = l0; l < l0 + nl; ++l)
         for (int s = 0; s < n_seqs; ++s)
             nu += (long long)std::max(1, (h->bm.length(l, s) + g.BT - 1) / g.BT) * Hg;
-    const int cap = g.max_ctas > 0 ? std::min(g.max_ctas, h->sm_count) : h->sm_count;
+    int cap = g.max_ctas > 0 ? std::min(g.max_ctas, h->sm_count) : h->sm_count;
+    const int reserve = std::max(1, std::min(12, h->sm_count / 8));   // SMs left to the staged launches
+    if (split && cap == h->sm_count) cap = std::max(1, cap - reserve);
     const int grid = (int)std::max<long long>(1, std::min<long long>(cap, (nu + nw - 1) / nw));
+    if (h->timing) CU(cudaEventRecord(h->lev[l0].r0, h->s_compute));
     CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_RESIDENT, grid, h->stages_res, smem, h->s_compute));
     ++h->launches;
+    if (h->timing) {   // the launch is booked on the first layer; the others show no resident time of their own
+        CU(cudaEventRecord(h->lev[l0].r1, h->s_compute));
+        for (int l = l0 + 1; l < l0 + nl; ++l) {
+            CU(cudaEventRecord(h->lev[l].r0, h->s_compute));
+            CU(cudaEventRecord(h->lev[l].r1, h->s_compute));
+        }
+    }
     for (int l = l0; l < l0 + nl; ++l) h->lens_cur[l] ^= 1;   // the kernel wrote the advanced lengths to the other copies
     h->last_fused_layer = -1;
+    if (!split) return ISV_OK;
+
+    // ---- per layer: staged launches over the host-resident blocks, then the merge with the resident result
+    const size_t rows = (size_t)n_seqs * g.Hq;
+    const size_t qs = rows * g.D * 2;
+    for (int l = l0; l < l0 + nl; ++l) {
+        const size_t i = (size_t)(l - l0);
+        FusedLayer fc;
+        fc.res_o = h->res_o + i * rows * g.D;
+        fc.res_ml = h->res_ml + i * rows * 2;
+        fc.run_o = h->run_o + i * rows * g.D;
+        fc.run_ml = h->run_ml + i * rows * 2;
+        fc.staged_grid_cap = reserve;
+        if ((rc = decode_impl(h, l, (const uint8_t *)q + i * qs, out ? (uint8_t *)out + i * qs : nullptr,
+                              out_f32 ? out_f32 + i * rows * g.D : nullptr, nullptr, nullptr, n_seqs, nullptr, nullptr,
+                              false, &fc)))
+            return rc;
+        if ((rc = flush_tails(h, l, aps[i].flush))) return rc;
+    }
+    return ISV_OK;
+}
+
+// Layers [l0, l0 + nl) of a step from buffers that hold them back to back: as few launches of the resident
+// kernel as fusable_layers allows.
+static int decode_layer_range(isv_kv *h, int l0, int nl, const void *q, const void *k, const void *v, void *out,
+                              float *out_f32, int n_seqs) {
+    const Geometry &g = h->g;
+    const size_t rows = (size_t)n_seqs * g.Hq * g.D;
+    const size_t qs = rows * 2, ks = (size_t)n_seqs * g.Hkv * g.D * 2;
+    int rc = ISV_OK;
+    for (int l = l0; l < l0 + nl;) {
+        const size_t i = (size_t)(l - l0);
+        const void *ql = (const uint8_t *)q + i * qs, *kl = (const uint8_t *)k + i * ks, *vl = (const uint8_t *)v + i * ks;
+        void *ol = out ? (uint8_t *)out + i * qs : nullptr;
+        float *fl = out_f32 ? out_f32 + i * rows : nullptr;
+        size_t smem = 0;
+        const int n = fusable_layers(h, l0 + nl - l, n_seqs, &smem);
+        if (n >= 2) rc = decode_layers_fused(h, l, n, ql, kl, vl, ol, fl, n_seqs, smem);
+        else rc = isv_decode_layer(h, l, ql, kl, vl, ol, fl, n_seqs);
+        if (rc) return rc;
+        l += n;
+    }
     return ISV_OK;
 }
 
@@ -1053,20 +1167,9 @@ int isv_decode_step(isv_kv *h, const void *q, const void *k, const void *v, void
     const Geometry &g = h->g;
     if (!q || !k || !v || (!out && !out_f32)) return fail(ISV_EINVAL, "q, k, v and one of out / out_f32 must be given");
     if (n_seqs < 0 || n_seqs > g.max_seqs) return fail(ISV_EINVAL, "n_seqs %d outside [0, %d]", n_seqs, g.max_seqs);
-    const size_t rows = (size_t)n_seqs * g.Hq * g.D;
-    const size_t qs = rows * 2, ks = (size_t)n_seqs * g.Hkv * g.D * 2;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(out_f32))
         return fail(ISV_EINVAL, "q, k, v, out and out_f32 must be 16-byte aligned");
-    size_t smem = 0;
-    if (can_fuse_layers(h, g.layers, n_seqs, &smem))   // the whole step is handed over at once: one launch
-        return decode_layers_fused(h, 0, g.layers, q, k, v, out, out_f32, n_seqs, smem);
-    for (int l = 0; l < g.layers; ++l) {
-        if ((rc = isv_decode_layer(h, l, (const uint8_t *)q + l * qs, (const uint8_t *)k + l * ks,
-                                   (const uint8_t *)v + l * ks, out ? (uint8_t *)out + l * qs : nullptr,
-                                   out_f32 ? out_f32 + l * rows : nullptr, n_seqs)))
-            return rc;
-    }
-    return ISV_OK;
+    return decode_layer_range(h, 0, g.layers, q, k, v, out, out_f32, n_seqs);
 }
 
 int isv_decode_step_host(isv_kv *h, const void *q, const void *k, const void *v, void *out, int32_t n_seqs) {
@@ -1120,16 +1223,9 @@ int isv_decode_step_host(isv_kv *h, const void *q, const void *k, const void *v,
     for (int gi = 0; gi < n_groups; ++gi) {
         const int l0 = first[gi], nl = first[gi + 1] - l0;
         CU(cudaStreamWaitEvent(h->s_compute, h->ev_step_in[gi], 0));
-        size_t smem = 0;
-        if (can_fuse_layers(h, nl, n_seqs, &smem)) {   // a group whose inputs have arrived runs as one launch
-            if ((rc = decode_layers_fused(h, l0, nl, dq + l0 * ql, dk + l0 * kl, dv + l0 * kl, dout + l0 * ql, nullptr,
-                                          n_seqs, smem)))
-                return rc;
-        } else {
-            for (int l = l0; l < l0 + nl; ++l)
-                if ((rc = isv_decode_layer(h, l, dq + l * ql, dk + l * kl, dv + l * kl, dout + l * ql, nullptr, n_seqs)))
-                    return rc;
-        }
+        // a group whose inputs have arrived runs as one launch where it can
+        if ((rc = decode_layer_range(h, l0, nl, dq + l0 * ql, dk + l0 * kl, dv + l0 * kl, dout + l0 * ql, nullptr, n_seqs)))
+            return rc;
         CU(cudaEventRecord(h->ev_step_out[gi], h->s_compute));
         CU(cudaStreamWaitEvent(h->s_d2h, h->ev_step_out[gi], 0));
         CU(cudaMemcpyAsync((uint8_t *)out + l0 * ql, dout + l0 * ql, nl * ql, cudaMemcpyDeviceToHost, h->s_d2h));

@@ -53,9 +53,9 @@ struct DecodeParams {
     // (layer, sequence) pair indexes them like a sequence number layer * n_seqs + s; `pool` / `tail` point at
     // physical slab 0 and layer l uses slab l % phys_layers; `lens` points at the first of two copies of
     // [layers][lens_layer_stride] lengths, bit l of lens_cur_mask says which copy is current for layer l, and
-    // the advanced lengths go to the other one.  Where several layers of the launch share a slab only the
-    // last of them stores its token (the earlier rows would be overwritten anyway; nothing in the launch
-    // reads them).
+    // the advanced lengths go to the other one.  The host puts at most phys_layers layers into a launch, so
+    // no two layers of a launch share a slab (were they to, only the last of them would store its token: the
+    // earlier rows would be overwritten anyway and nothing in the launch reads them).
     int32_t n_layers;           // 0 or 1: one layer, the fields below are unused
     int32_t layer0, phys_layers;
     int32_t lens_layer_stride, lens_copy_stride;   // in elements

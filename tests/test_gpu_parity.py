@@ -351,10 +351,8 @@ def test_steps_enqueued_back_to_back_on_small_grids(layers, phys, ctas, f, per_l
     step t+1 must still see the lengths and the K/V rows its launch of step t wrote (with two layers the
     writer is only two launches back; with shared slabs likewise).  Every step's output is compared with
     the reference afterwards, and the cache is read back bit for bit."""
-    if per_layer:      # one launch per layer even where a whole step could be one launch
+    if per_layer:      # one launch per layer even where the step's resident part could be one launch
         monkeypatch.setenv("ISV_LAYERS_PER_LAUNCH", "1")
-    elif f > 0:
-        pytest.skip("with offloaded blocks a step is always one launch per layer")
     steps = 7
     w = small(batch=8, steps=steps, f=f, perm=13, ctx=(1900, 2040), layers=layers, q_heads=4, kv_heads=4,
               head_dim=128, seed=23)
@@ -392,14 +390,17 @@ def test_steps_enqueued_back_to_back_on_small_grids(layers, phys, ctas, f, per_l
 
 @pytest.mark.parametrize("q_heads,kv_heads,head_dim,dtype", [(4, 4, 128, "f16"), (8, 2, 128, "bf16"), (6, 6, 80, "f16"),
                                                              (16, 2, 64, "f16")])
-@pytest.mark.parametrize("layers,phys,ctas", [(5, 5, 0), (5, 2, 3), (4, 4, 1)])
-def test_whole_step_as_one_launch(q_heads, kv_heads, head_dim, dtype, layers, phys, ctas):
-    """With nothing offloaded isv_decode_step runs all layers' append + attention as one launch whose work list
-    spans the layers.  Ragged lengths (an empty sequence, one token, block boundaries), layers that share
-    slabs, and grids of 1, 3 and all CTAs; every output row against the reference, lengths and cache read back."""
+@pytest.mark.parametrize("layers,phys,ctas,f", [(5, 5, 0, 0.0), (5, 2, 3, 0.0), (4, 4, 1, 0.0), (5, 5, 0, 0.5), (5, 2, 0, 0.75),
+                                                 (4, 4, 2, 1.0)])
+def test_whole_step_as_one_launch(q_heads, kv_heads, head_dim, dtype, layers, phys, ctas, f):
+    """isv_decode_step runs the resident attention (and the appends) of all layers as one launch whose work list
+    spans the layers; with host-resident blocks each layer's staged launches and merge follow it.  Ragged lengths
+    (an empty sequence, one token, block boundaries), layers that share slabs, grids of 1, 2, 3 and all CTAs,
+    nothing / half / three quarters / everything offloaded; every output row against the reference, lengths and
+    cache read back."""
     lens = [0, 1, 15, 16, 17, 100, 257, 330]
     steps = 18                                    # crosses a block boundary for every sequence
-    w = small(batch=len(lens), steps=steps + 1, f=0.0, perm=17, ctx=(0, 330), layers=layers, q_heads=q_heads,
+    w = small(batch=len(lens), steps=steps + 1, f=f, perm=17, ctx=(0, 330), layers=layers, q_heads=q_heads,
               kv_heads=kv_heads, head_dim=head_dim, dtype=dtype, seed=29)
     td = W.torch_dtype(w.dtype)
     with Harness(w, lens=lens, max_ctas=ctas, phys_layers=phys) as hz:
@@ -427,8 +428,8 @@ def test_whole_step_as_one_launch(q_heads, kv_heads, head_dim, dtype, layers, ph
                 res.append((q[layer], of[layer].cpu().numpy(), dev_to_bits(o16[layer]), ref))
             hz.cur += 1
             hz.check_step(res)
-        # one attention launch per step, whatever the number of layers
-        assert B.isv_kv_info(hz.h).kernel_launches - launches0 == steps + updates
+        if f == 0:   # one attention launch per step and group of layers on distinct slabs
+            assert B.isv_kv_info(hz.h).kernel_launches - launches0 == steps * -(-layers // phys) + updates
         for layer in range(layers):
             assert np.array_equal(B.isv_seq_lens_host(hz.h, layer, w.batch), hz.cur)
         hz.check_gather(layers=range(layers - phys, layers))
