@@ -1186,16 +1186,18 @@ int isv_decode_step_host(isv_kv *h, const void *q, const void *k, const void *v,
     uint8_t *dq = h->step_buf, *dout = dq + qs_max, *dk = dout + qs_max, *dv = dk + ks_max;
     // Inputs travel in groups of layers on their own stream and results go back on the write-back stream,
     // so that only the first group's copy and the last group's read-back are not hidden behind the attention
-    // of the other layers.  Those two groups are a single layer; in between the groups grow to eight layers
-    // (every group boundary is a cross-stream wait, which costs the launch overlap between two layers).
+    // of the other layers.  Those two groups are a single layer; in between the groups grow fourfold (a layer's
+    // inputs cross the link several times faster than its attention runs, so the copies stay ahead), because
+    // every group boundary is a cross-stream wait and ends a launch.
     std::vector<int> first;   // first layer of each group, and the end
     {
-        int l = 0;
-        const int head[2] = {1, 3};
-        for (int i = 0; i < 2 && l < g.layers; ++i) { first.push_back(l); l += std::min(head[i], g.layers - l); }
-        while (g.layers - l > 9) { first.push_back(l); l += 8; }
-        if (g.layers - l > 1) { first.push_back(l); l = g.layers - 1; }
-        if (l < g.layers) { first.push_back(l); l = g.layers; }
+        int l = 0, n = 1;
+        while (l < g.layers - 1) {
+            first.push_back(l);
+            l += std::min(n, g.layers - 1 - l);
+            n *= 4;
+        }
+        first.push_back(l);           // the last layer on its own
         first.push_back(g.layers);
     }
     const int n_groups = (int)first.size() - 1;
