@@ -297,6 +297,11 @@ int isv_sync(isv_kv *h, uint32_t *status_out);
 
 /* ---- failure handling ----------------------------------------------------- */
 
+/* (The paper treats only predicted out-of-memory, Algorithm 1's "Unsuitable" case, which isv_kv_alloc's
+ * ISV_ENOMEM_* codes mirror; it has no counterpart for what follows.  These calls keep a lost transfer or
+ * a stuck stream from turning into a hang: every wait of the library, on the device and on the host, can
+ * be given a limit, and running into it is reported as a status or an error code with the handle intact.) */
+
 /* Limit, in seconds, of every host-side wait of this handle (isv_sync, isv_step_timing, isv_kv_fill,
  * isv_fill_timing, isv_kv_gather, isv_decode_step_host): a wait that exceeds it returns ISV_ETIMEOUT
  * and leaves the work enqueued, so the caller can wait again, report, or tear down.  0 (the default)

@@ -437,6 +437,55 @@ def test_whole_step_as_one_launch(q_heads, kv_heads, head_dim, dtype, layers, ph
         hz.check_step(hz.step(fused=True))
 
 
+@pytest.mark.parametrize("f,phys", [(0.0, 6), (0.0, 2), (0.5, 6), (0.75, 3)])
+def test_host_buffer_step_equals_device_buffer_step(f, phys):
+    """isv_decode_step_host copies the inputs in groups of layers (1, 4, 1 of six) and runs each group as soon as
+    it has arrived, the middle one as fused launches: the same result as isv_decode_step on device buffers up to
+    the summation order, and both within the bound of the reference."""
+    layers, steps = 6, 5
+    lens = [40, 200, 17, 333, 64]
+    w = small(batch=len(lens), steps=steps, f=f, perm=19, ctx=(17, 333), layers=layers, q_heads=8, kv_heads=4,
+              head_dim=128, seed=37)
+    td = W.torch_dtype(w.dtype)
+    with Harness(w, lens=lens, phys_layers=phys) as ha, Harness(w, lens=lens, phys_layers=phys) as hb:
+        ha.fill()
+        hb.fill()
+        for t in range(steps):
+            ks, vs, qs = zip(*[W.host_step(w, ha.rng) for _ in range(layers)])
+            for _ in range(layers):
+                W.host_step(w, hb.rng)
+            k, v, q = (np.stack(x) for x in (ks, vs, qs))
+            kd, vd, qd = (bits_to_dev(x, w.dtype) for x in (k, v, q))
+            od = torch.zeros((layers, w.batch, w.q_heads, w.head_dim), device="cuda", dtype=td)
+            of = torch.full((layers, w.batch, w.q_heads, w.head_dim), float("nan"), device="cuda")
+            torch.cuda.synchronize()
+            B.isv_decode_step(ha.h, qd, kd, vd, od, of, w.batch)
+            assert B.isv_sync(ha.h) == 0
+            kp, vp, qp = (torch.from_numpy(x.view(np.int16)).pin_memory() for x in (k, v, q))
+            op = torch.zeros((layers, w.batch, w.q_heads, w.head_dim), dtype=torch.int16).pin_memory()
+            B.isv_decode_step_host(hb.h, qp, kp, vp, op, w.batch)
+            got_host = op.numpy().view(np.uint16)
+            # the two paths cut the work differently (other launch groups), so sums may differ in the last bits
+            diff = np.abs(oa.to_f64(values(got_host, w.dtype)) - oa.to_f64(values(dev_to_bits(od), w.dtype)))
+            assert float(diff.max()) <= 2.0 ** -10
+            res, res_host = [], []
+            for layer in range(layers):
+                if phys < layers:
+                    ha.shadow.store_at(layer % phys, k[layer], v[layer], ha.cur.tolist())
+                    ref = ha.reference(layer, q[layer], lens=ha.cur + 1)
+                else:
+                    ha.shadow.append(layer, k[layer], v[layer])
+                    ref = None
+                res.append((q[layer], of[layer].cpu().numpy(), dev_to_bits(od[layer]), ref))
+                res_host.append((q[layer], None, got_host[layer], ref if ref is not None else ha.reference(layer, q[layer])))
+            ha.cur += 1
+            ha.check_step(res)
+            ha.check_step(res_host)
+        assert B.isv_sync(hb.h) == 0
+        hb.shadow, hb.cur = ha.shadow, ha.cur            # same inputs went into both caches
+        hb.check_gather(layers=range(layers - phys, layers))
+
+
 def test_device_lengths_beyond_the_table_row_are_clamped_and_flagged():
     """Caller-supplied device lengths are not trusted: one that exceeds what a table row covers (or is
     negative) is clamped, the status word says so, and the other sequences are unaffected."""
