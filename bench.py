@@ -10,8 +10,8 @@ attention per layer).  One JSON line is printed by rank 0.
 The default workload is the offload sweep the metric is named after: the
 13B-shaped ragged batch (c5) at offload fractions 0 / 0.25 / 0.5 / 0.75 / 1, the
 7B-shaped batches with nothing (c2) and half (c3) of the cache offloaded, the
-8B-GQA batch with three quarters offloaded (c4) and the paper's own OPT-2.7B
-offline shape.  The headline figures (`value`, `config`, `roofline`, `e2e`) are
+8B-GQA batch with three quarters (c4) and nothing offloaded, and the paper's
+own OPT-2.7B offline shape.  The headline figures (`value`, `config`, `roofline`, `e2e`) are
 those of c5 at offload fraction 0.5, timed for exactly --steps steps after
 --warmup warm-up steps; every other point is listed under `sweep` with its own
 step counts, its tokens/s, its fraction of the combined HBM / host-link
@@ -183,6 +183,7 @@ def sweep_points(K, Wm, layers=None, batch=None):
            (C["opt2.7b"], 120, max(3, min(Wm, 8)), 3, True),
            (C["c3"], 4, 3, 1, False),
            (C["c4"], 4, 3, 1, False),
+           (C["c4"].with_(offload_frac=0.0), 9, 3, 3, False),     # the grouped-query (tensor-core) variant at the HBM rate
            (C["c5"].with_(offload_frac=0.0), 9, 3, 3, False)]
     for f in (0.25, 0.5, 0.75, 1.0):
         if ("c5", f) == HEADLINE:
@@ -193,9 +194,9 @@ def sweep_points(K, Wm, layers=None, batch=None):
     return [(w.with_(**over), k_pt, w_pt, reps, reset) for (w, k_pt, w_pt, reps, reset) in pts]
 
 
-def choose_phys_layers(w, max_tokens, requested):
-    """Physical KV slabs to hold: as many as fit a budget (0.7 of free HBM; 24 GiB or a third of the
-    available host memory for the pinned pool), at most `layers`.  Every slab is far larger than L2."""
+def choose_phys_layers(w, max_tokens, requested, local_ranks=1):
+    """Physical KV slabs to hold: as many as fit a budget (0.7 of free HBM; 24 GiB or this rank's share of a
+    third of the available host memory for the pinned pool), at most `layers`.  Every slab is far larger than L2."""
     if requested:
         return requested
     import torch
@@ -213,7 +214,7 @@ def choose_phys_layers(w, max_tokens, requested):
                 avail = int(ln.split()[1]) * 1024
     except OSError:
         pass
-    host_budget = min(0.35 * avail, 24 << 30)
+    host_budget = min(0.35 * avail / max(1, local_ranks), 24 << 30)
     p = w.layers
     if hbm_layer:
         p = min(p, int(hbm_budget // hbm_layer))
@@ -359,7 +360,7 @@ def measure_point(cx: Ctx, w, K, Wm, reps, reset_between, want_e2e, phys_req=0):
     total_steps = (Wm + K) if reset_between else (Wm + reps * K)
     max_tokens = w.ctx_max + total_steps + extra + 1
     lens = W.prompt_lens(w)
-    phys = choose_phys_layers(w, max_tokens, phys_req)
+    phys = choose_phys_layers(w, max_tokens, phys_req, cx.world)
     t_alloc = time.perf_counter()
     h = B.isv_kv_alloc(**B.desc_from_workload(w, phys_layers=phys, max_tokens_per_seq=max_tokens,
                                               compute_stream=stream.cuda_stream))
