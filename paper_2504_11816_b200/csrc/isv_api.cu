@@ -198,10 +198,10 @@ int dev_alloc(void **p, size_t bytes, uint64_t *tally, const char *what) {
 // Ring depth per warp: the default depth (or ISV_DECODE_STAGES, a tuning knob), reduced until it fits.
 int pick_stages(const Geometry &g, int mode, int smem_limit, size_t *smem_out) {
     int best = 0;
-    int cap = decode_default_stages(g.D, g.BT, g.GT);
+    int cap = decode_default_stages(g.D, g.BT, g.GT, g.HP);
     if (const char *e = getenv("ISV_DECODE_STAGES")) cap = std::max(2, std::min(12, atoi(e)));
     for (int st = 2; st <= cap; ++st) {
-        const size_t b = decode_smem_bytes(g.D, g.BT, g.GT, st, g.max_seqs, mode);
+        const size_t b = decode_smem_bytes(g.D, g.BT, g.GT, g.HP, st, g.max_seqs, mode);
         if (b <= (size_t)smem_limit) { best = st; *smem_out = b; }
     }
     return best;
@@ -436,8 +436,8 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
         return bail(fail(ISV_EINVAL, "shared memory (%d bytes) too small for this shape", smem_limit));
     const bool bf16 = g.dtype == ISV_BF16;
     // the per-function limit is shared by all handles: always raise it to the device maximum
-    CUB(decode_configure(g.D, g.GT, g.BT, bf16, MODE_RESIDENT, (size_t)smem_limit));
-    CUB(decode_configure(g.D, g.GT, g.BT, bf16, MODE_STAGED, (size_t)smem_limit));
+    CUB(decode_configure(g.D, g.GT, g.HP, g.BT, bf16, MODE_RESIDENT, (size_t)smem_limit));
+    CUB(decode_configure(g.D, g.GT, g.HP, g.BT, bf16, MODE_STAGED, (size_t)smem_limit));
 
     if (desc->compute_stream) {
         h->s_compute = (cudaStream_t)desc->compute_stream;
@@ -480,7 +480,7 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
     // scratch
     const size_t rows = (size_t)g.max_seqs * g.Hq;
     const int max_grid = g.max_ctas > 0 ? std::min(g.max_ctas, h->sm_count) : h->sm_count;
-    const size_t slots = 2ull * max_grid * decode_warps(g.GT, g.D) * g.GT;   // two partials per warp and query head
+    const size_t slots = 2ull * max_grid * decode_warps(g.GT, g.D, g.HP) * g.GT;   // two partials per warp and query head
     if ((rc = dev_alloc((void **)&h->part_o, slots * g.D * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
     if ((rc = dev_alloc((void **)&h->part_ml, slots * 2 * 4, &h->scratch_bytes, "split partials"))) return bail(rc);
     // one arrival counter per (layer, sequence, head group): a launch that covers several layers uses them all
@@ -491,7 +491,7 @@ int isv_kv_alloc(isv_kv **out, const isv_kv_desc *desc) {
         // per-layer results then wait for the layers' offloaded parts), else one; a launch covers at most
         // phys_layers layers
         if (g.phys_layers > 1 && g.layers <= 64 &&
-            decode_smem_bytes(g.D, g.BT, g.GT, h->stages_res, 2 * g.max_seqs, MODE_RESIDENT) <= (size_t)smem_limit)
+            decode_smem_bytes(g.D, g.BT, g.GT, g.HP, h->stages_res, 2 * g.max_seqs, MODE_RESIDENT) <= (size_t)smem_limit)
             h->res_layers = g.phys_layers;
         const size_t nl = (size_t)h->res_layers;
         if ((rc = dev_alloc((void **)&h->res_o, nl * rows * g.D * 4, &h->scratch_bytes, "resident result"))) return bail(rc);
@@ -807,8 +807,8 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
         return fail(ISV_EINVAL, "q, out and out_f32 must be 16-byte aligned");
     if (n_seqs == 0) return ISV_OK;
     const bool bf16 = g.dtype == ISV_BF16;
-    const int Hg = g.Hkv * g.P;
-    const int nw = decode_warps(g.GT, g.D);
+    const int Hg = g.groups();
+    const int nw = decode_warps(g.GT, g.D, g.HP);
     const OffPlan &pl = h->bm.plan(layer, n_seqs, h->zero_copy ? (1 << 30) : g.chunk_blocks);
     const bool offloaded = !pl.chunks.empty();
     const int phys = layer % g.phys_layers;
@@ -888,7 +888,7 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
             // reading in place needs few CTAs to saturate the link and leaves the other SMs to the resident kernel
             const long long cap2 = h->zero_copy ? std::max(1, h->sm_count / 4) : (fc ? fc->staged_grid_cap : h->sm_count);
             const int grid = (int)std::max<long long>(1, std::min<long long>(cap2, (nu2 + nw - 1) / nw));
-            CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_STAGED, grid, h->stages_stg, h->smem_stg, h->s_off));
+            CU(launch_decode(p, g.D, g.GT, g.HP, g.BT, bf16, MODE_STAGED, grid, h->stages_stg, h->smem_stg, h->s_off));
             ++h->launches;
             if (r >= 0) {
                 CU(cudaEventRecord(h->ev_freed[r], h->s_off));
@@ -936,7 +936,7 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
             p.drop_first_copy = 1;
         }
         if (le) CU(cudaEventRecord(le->r0, h->s_compute));
-        CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_RESIDENT, grid, h->stages_res, h->smem_res, h->s_compute));
+        CU(launch_decode(p, g.D, g.GT, g.HP, g.BT, bf16, MODE_RESIDENT, grid, h->stages_res, h->smem_res, h->s_compute));
         ++h->launches;
         if (le) CU(cudaEventRecord(le->r1, h->s_compute));
         if (k_new) h->lens_cur[layer] ^= 1;   // the kernel wrote the advanced lengths to the other copy
@@ -1010,10 +1010,10 @@ static int fusable_layers(const isv_kv *h, int nl, int n_seqs, size_t *smem) {
         if (h->zero_copy || h->res_layers < 2) return 1;
         nl = std::min(nl, h->res_layers);
     }
-    while (nl >= 2 && decode_smem_bytes(g.D, g.BT, g.GT, h->stages_res, nl * n_seqs, MODE_RESIDENT) > (size_t)h->smem_limit)
+    while (nl >= 2 && decode_smem_bytes(g.D, g.BT, g.GT, g.HP, h->stages_res, nl * n_seqs, MODE_RESIDENT) > (size_t)h->smem_limit)
         --nl;
     if (nl < 2) return 1;
-    *smem = decode_smem_bytes(g.D, g.BT, g.GT, h->stages_res, nl * n_seqs, MODE_RESIDENT);
+    *smem = decode_smem_bytes(g.D, g.BT, g.GT, g.HP, h->stages_res, nl * n_seqs, MODE_RESIDENT);
     return nl;
 }
 
@@ -1065,8 +1065,8 @@ static int decode_layers_fused(isv_kv *h, int l0, int nl, const void *q, const v
     }
 
     const bool bf16 = g.dtype == ISV_BF16;
-    const int Hg = g.Hkv * g.P;
-    const int nw = decode_warps(g.GT, g.D);
+    const int Hg = g.groups();
+    const int nw = decode_warps(g.GT, g.D, g.HP);
     DecodeParams p{};
     p.table = h->table_dev;
     p.table_stride = g.NB;
@@ -1104,7 +1104,7 @@ static int decode_layers_fused(isv_kv *h, int l0, int nl, const void *q, const v
     if (split && cap == h->sm_count) cap = std::max(1, cap - reserve);
     const int grid = (int)std::max<long long>(1, std::min<long long>(cap, (nu + nw - 1) / nw));
     if (h->timing) CU(cudaEventRecord(h->lev[l0].r0, h->s_compute));
-    CU(launch_decode(p, g.D, g.GT, g.BT, bf16, MODE_RESIDENT, grid, h->stages_res, smem, h->s_compute));
+    CU(launch_decode(p, g.D, g.GT, g.HP, g.BT, bf16, MODE_RESIDENT, grid, h->stages_res, smem, h->s_compute));
     ++h->launches;
     if (h->timing) {   // the launch is booked on the first layer; the others show no resident time of their own
         CU(cudaEventRecord(h->lev[l0].r1, h->s_compute));

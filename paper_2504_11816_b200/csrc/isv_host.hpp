@@ -24,6 +24,8 @@ struct Geometry {
     int G = 0;                     // query heads per KV head
     int GT = 0;                    // query heads handled together by one warp
     int P = 0;                     // passes over a KV head = G / GT
+    int HP = 1;                    // KV heads per head group (2: two adjacent heads of a multi-head shape per visit)
+    int groups() const { return Hkv * P / HP; }   // head groups per sequence
     int max_ctas = 0;              // cap on the decode kernel's grid (0 = one CTA per SM)
     uint32_t tile_bytes = 0;       // one (block, K|V, head) tile
     uint64_t block_bytes = 0;      // 2 * Hkv * tile_bytes
@@ -271,8 +273,9 @@ inline const char *make_geometry(const isv_kv_desc &d, Geometry *out) {
     g.Hq = d.q_heads;
     g.Hkv = d.kv_heads;
     g.G = g.Hq / g.Hkv;
-    g.GT = group_heads(g.G);
-    g.P = g.G / g.GT;
+    g.HP = pair_heads(g.G, d.head_dim, g.Hkv);
+    g.GT = g.HP == 2 ? 2 : group_heads(g.G);
+    g.P = g.HP == 2 ? 1 : g.G / g.GT;
     if (d.head_dim != 64 && d.head_dim != 80 && d.head_dim != 128) return "head_dim must be 64, 80 or 128";
     g.D = d.head_dim;
     if (d.block_tokens != 16) return "block_tokens must be 16";

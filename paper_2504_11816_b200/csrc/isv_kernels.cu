@@ -157,46 +157,39 @@ __device__ __forceinline__ int tail_token(int grp, int sub) {
     return 4 * pi + ((grp + pi) & 3);
 }
 
-// Scores of the tile's tokens against the GT query heads (log2 domain, q is
-// pre-scaled), and the running maximum brought up to date (o and l rescaled).
-template <int D, int GT, int BT, bool BF16>
+// Scores of the tokens of GT K tiles, one per query head (head g's tile is sK + g * TSTRIDE), in the log2
+// domain (q is pre-scaled), and the running maxima brought up to date (o and l rescaled).
+template <int D, int GT, int BT, bool BF16, int TSTRIDE>
 __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp, int sub,
                                             const float (&q)[GT][(D + 63) / 64 * 8], float (&sc)[BT / 4][GT],
                                             float (&o)[GT][(D + 63) / 64 * 8], float (&m)[GT], float (&l)[GT]) {
     constexpr int NVF = D / 64, NV = (D + 63) / 64, NQ = BT / 4, ROW = D * 2;
     static_assert(D % 64 == 0 || D % 64 == 16, "head_dim: whole 64-element spans, plus at most a 16-element tail");
 #pragma unroll
-    for (int i = 0; i < NQ; ++i) {
-        const int t = 4 * i + grp;
-        const uint4 *krow = reinterpret_cast<const uint4 *>(sK + t * ROW);
-        float a0[GT], a1[GT];   // two chains per dot product
+    for (int g = 0; g < GT; ++g) {
+        const uint8_t *tile = sK + g * TSTRIDE;
 #pragma unroll
-        for (int g = 0; g < GT; ++g) a0[g] = a1[g] = 0.f;
+        for (int i = 0; i < NQ; ++i) {
+            const int t = 4 * i + grp;
+            const uint4 *krow = reinterpret_cast<const uint4 *>(tile + t * ROW);
+            float a0 = 0.f, a1 = 0.f;   // two chains per dot product
 #pragma unroll
-        for (int v = 0; v < NVF; ++v) {
-            float kf[8];
-            cvt8<BF16>(krow[swz(v * 8 + sub, t, D / 8)], kf);
+            for (int v = 0; v < NVF; ++v) {
+                float kf[8];
+                cvt8<BF16>(krow[swz(v * 8 + sub, t, D / 8)], kf);
 #pragma unroll
-            for (int g = 0; g < GT; ++g)
-#pragma unroll
-                for (int e = 0; e < 8; e += 2)
-                    ffma2(a0[g], a1[g], q[g][v * 8 + e], q[g][v * 8 + e + 1], kf[e], kf[e + 1]);
-        }
-#pragma unroll
-        for (int g = 0; g < GT; ++g) {
-            float a = a0[g] + a1[g];
+                for (int e = 0; e < 8; e += 2) ffma2(a0, a1, q[g][v * 8 + e], q[g][v * 8 + e + 1], kf[e], kf[e + 1]);
+            }
+            float a = a0 + a1;
             a += __shfl_xor_sync(kFull, a, 4);
             a += __shfl_xor_sync(kFull, a, 2);
             a += __shfl_xor_sync(kFull, a, 1);
             sc[i][g] = a;
         }
-    }
-    if (NV > NVF) {   // the 16-element tails, one chunk per lane (token assignment: see tail_token)
-        const int tt = tail_token(grp, sub);
-        float kf[8];
-        cvt8<BF16>(reinterpret_cast<const uint4 *>(sK + tt * ROW)[NVF * 8 + (sub & 1)], kf);
-#pragma unroll
-        for (int g = 0; g < GT; ++g) {
+        if (NV > NVF) {   // the 16-element tails, one chunk per lane (token assignment: see tail_token)
+            const int tt = tail_token(grp, sub);
+            float kf[8];
+            cvt8<BF16>(reinterpret_cast<const uint4 *>(tile + tt * ROW)[NVF * 8 + (sub & 1)], kf);
             float tp = 0.f, tp1 = 0.f;
 #pragma unroll
             for (int e = 0; e < 8; e += 2) ffma2(tp, tp1, q[g][NVF * 8 + e], q[g][NVF * 8 + e + 1], kf[e], kf[e + 1]);
@@ -230,47 +223,42 @@ __device__ __forceinline__ void tile_scores(const uint8_t *sK, int ntok, int grp
     }
 }
 
-// o += softmax weights x V for the tile whose scores are in sc.
-template <int D, int GT, int BT, bool BF16>
+// o += softmax weights x V for the GT V tiles (head g's tile is sV + g * TSTRIDE) whose scores are in sc.
+template <int D, int GT, int BT, bool BF16, int TSTRIDE>
 __device__ __forceinline__ void tile_values(const uint8_t *sV, int ntok, int grp, int sub,
                                             const float (&sc)[BT / 4][GT], float (&o)[GT][(D + 63) / 64 * 8],
                                             const float (&m)[GT], float (&l)[GT]) {
     constexpr int NVF = D / 64, NV = (D + 63) / 64, NQ = BT / 4, ROW = D * 2;
-    float pwv[NQ][GT];   // the weights of the four passes (used again by the tail step)
 #pragma unroll
-    for (int i = 0; i < NQ; ++i) {
-        const int t = 4 * i + grp;
+    for (int g = 0; g < GT; ++g) {
+        const uint8_t *tile = sV + g * TSTRIDE;
+        float pwv[NQ];   // the weights of the four passes (used again by the tail step)
 #pragma unroll
-        for (int g = 0; g < GT; ++g) pwv[i][g] = 0.f;
-        if (t < ntok) {   // slots past the sequence end hold unspecified bits: never touch them
+        for (int i = 0; i < NQ; ++i) {
+            const int t = 4 * i + grp;
+            pwv[i] = 0.f;
+            if (t < ntok) {   // slots past the sequence end hold unspecified bits: never touch them
+                pwv[i] = fast_exp2(sc[i][g] - m[g]);
+                l[g] += pwv[i];
+                const uint4 *vrow = reinterpret_cast<const uint4 *>(tile + t * ROW);
 #pragma unroll
-            for (int g = 0; g < GT; ++g) {
-                pwv[i][g] = fast_exp2(sc[i][g] - m[g]);
-                l[g] += pwv[i][g];
-            }
-            const uint4 *vrow = reinterpret_cast<const uint4 *>(sV + t * ROW);
-#pragma unroll
-            for (int v = 0; v < NVF; ++v) {
-                float vf[8];
-                cvt8<BF16>(vrow[swz(v * 8 + sub, t, D / 8)], vf);
-#pragma unroll
-                for (int g = 0; g < GT; ++g)
+                for (int v = 0; v < NVF; ++v) {
+                    float vf[8];
+                    cvt8<BF16>(vrow[swz(v * 8 + sub, t, D / 8)], vf);
 #pragma unroll
                     for (int e = 0; e < 8; e += 2)
-                        ffma2(o[g][v * 8 + e], o[g][v * 8 + e + 1], pwv[i][g], pwv[i][g], vf[e], vf[e + 1]);
+                        ffma2(o[g][v * 8 + e], o[g][v * 8 + e + 1], pwv[i], pwv[i], vf[e], vf[e + 1]);
+                }
             }
         }
-    }
-    if (NV > NVF) {
-        // The V tails stay with the group that owns the token: their products are added to that group's
-        // accumulators, which are scaled by that group's running maximum (no rotation as for the K tails).
-        const int pi = sub >> 1, tt = 4 * pi + grp;
-        if (tt < ntok) {
-            float vf[8];
-            cvt8<BF16>(reinterpret_cast<const uint4 *>(sV + tt * ROW)[NVF * 8 + (sub & 1)], vf);
-#pragma unroll
-            for (int g = 0; g < GT; ++g) {
-                const float pw = pi == 0 ? pwv[0][g] : pi == 1 ? pwv[1][g] : pi == 2 ? pwv[2][g] : pwv[3][g];
+        if (NV > NVF) {
+            // The V tails stay with the group that owns the token: their products are added to that group's
+            // accumulators, which are scaled by that group's running maximum (no rotation as for the K tails).
+            const int pi = sub >> 1, tt = 4 * pi + grp;
+            if (tt < ntok) {
+                float vf[8];
+                cvt8<BF16>(reinterpret_cast<const uint4 *>(tile + tt * ROW)[NVF * 8 + (sub & 1)], vf);
+                const float pw = pi == 0 ? pwv[0] : pi == 1 ? pwv[1] : pi == 2 ? pwv[2] : pwv[3];
 #pragma unroll
                 for (int e = 0; e < 8; e += 2)
                     ffma2(o[g][NVF * 8 + e], o[g][NVF * 8 + e + 1], pw, pw, vf[e], vf[e + 1]);
@@ -309,7 +297,9 @@ __device__ __forceinline__ void store_row_grouped(void *out, float *out_f32, siz
 //
 // The decode kernel is written once; what a warp does with a K tile, a V tile, this step's token and
 // its finished (m, l, o) state comes from one of two classes:
-//   ScalarMath  CUDA-core arithmetic, GT query heads per KV tile (used for GT = 1, multi-head attention)
+//   ScalarMath  CUDA-core arithmetic for multi-head attention: one query head per KV head.  A visit may
+//               carry the tiles of HP = 2 adjacent KV heads (they are contiguous in a block), each with its
+//               own query head: at head_dim 64 and 80 that halves the per-visit bookkeeping per byte
 //   MmaMath     tensor-core arithmetic (mma.sync m16n8k16, fp32 accumulation) for grouped-query
 //               attention: the 2..16 query heads that share a KV head are the rows of one 16-row
 //               operand, so a KV tile is read once for all of them
@@ -319,6 +309,8 @@ __device__ __forceinline__ void store_row_grouped(void *out, float *out_f32, siz
 template <int D_, int GT_, int BT_, bool BF16_>
 struct ScalarMath {
     static constexpr int D = D_, BT = BT_, NVF = D_ / 64, NV = (D_ + 63) / 64, E = NV * 8;   // 8 elements per span and lane
+    static constexpr int HP = GT_;            // KV heads (tiles) per visit: query head g of the group reads tile g
+    static constexpr int TILE1 = BT_ * D_ * 2;
     static constexpr bool BF16 = BF16_;
     float q[GT_][E], o[GT_][E], m[GT_], l[GT_], sc[BT_ / 4][GT_];
     int grp, sub;
@@ -351,13 +343,13 @@ struct ScalarMath {
         }
     }
     __device__ __forceinline__ void k_tile(const uint8_t *tile, int ntok) {
-        tile_scores<D, GT_, BT, BF16>(tile, ntok, grp, sub, q, sc, o, m, l);
+        tile_scores<D, GT_, BT, BF16, TILE1>(tile, ntok, grp, sub, q, sc, o, m, l);
     }
     __device__ __forceinline__ void v_tile(const uint8_t *tile, int ntok) {
-        tile_values<D, GT_, BT, BF16>(tile, ntok, grp, sub, sc, o, m, l);
+        tile_values<D, GT_, BT, BF16, TILE1>(tile, ntok, grp, sub, sc, o, m, l);
     }
-    // This step's token, read from the caller's rows: all groups compute its scores (the shuffles
-    // need every lane), group 0 keeps it.
+    // This step's token, read from the caller's rows (head g's rows are krow + g * D, vrow + g * D): all
+    // groups compute its scores (the shuffles need every lane), group 0 keeps it.
     __device__ __forceinline__ void new_token(const uint16_t *krow, const uint16_t *vrow) {
         float a[GT_];
 #pragma unroll
@@ -365,12 +357,13 @@ struct ScalarMath {
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             if (v * 64 + sub * 8 >= D) continue;   // the tail is counted once: by lanes sub 0 and 1
-            float kf[8];
-            cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(krow + v * 64 + sub * 8)), kf);
 #pragma unroll
-            for (int g = 0; g < GT_; ++g)
+            for (int g = 0; g < GT_; ++g) {
+                float kf[8];
+                cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(krow + g * D + v * 64 + sub * 8)), kf);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) a[g] = fmaf(q[g][v * 8 + e], kf[e], a[g]);
+            }
         }
 #pragma unroll
         for (int g = 0; g < GT_; ++g) {
@@ -395,12 +388,13 @@ struct ScalarMath {
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
                 if (v * 64 + sub * 8 >= D) continue;
-                float vf[8];
-                cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(vrow + v * 64 + sub * 8)), vf);
 #pragma unroll
-                for (int g = 0; g < GT_; ++g)
+                for (int g = 0; g < GT_; ++g) {
+                    float vf[8];
+                    cvt8<BF16>(__ldg(reinterpret_cast<const uint4 *>(vrow + g * D + v * 64 + sub * 8)), vf);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) o[g][v * 8 + e] = fmaf(pw[g], vf[e], o[g][v * 8 + e]);
+                }
             }
         }
     }
@@ -530,6 +524,7 @@ __device__ __forceinline__ float2 unpack2(uint32_t w) {
 template <int D_, bool BF16_>
 struct MmaMath {
     static constexpr int D = D_, BT = 16, ROW = D_ * 2;
+    static constexpr int HP = 1;              // one KV head (tile) per visit, shared by the group's query heads
     static constexpr bool BF16 = BF16_;
     uint32_t qa[D_ / 16][4];    // Q as A fragments, one per 16 dims
     float oacc[D_ / 8][4];      // O accumulators: [j][0..1] row r, [j][2..3] row r + 8, dims 8 j + 2 c, + 1
@@ -957,7 +952,9 @@ template <class Math, int MODE, int NW>
 __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p, const int stages) {
     constexpr int D = Math::D, BT = Math::BT;
     constexpr bool BF16 = Math::BF16;
-    constexpr uint32_t TILE = BT * D * 2;
+    constexpr int HP = Math::HP;                 // KV heads whose tiles one visit carries (adjacent in a block)
+    constexpr uint32_t TILE1 = BT * D * 2;       // one (block, K|V, head) tile
+    constexpr uint32_t TILE = TILE1 * HP;        // what a ring slot holds and one bulk copy brings
     extern __shared__ __align__(128) uint8_t smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     Math mth;
@@ -993,9 +990,9 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
     }
     const uint32_t spin_limit = p.spin_limit ? p.spin_limit : kSpinLimit;
 
-    const int Hg = p.Hkv * p.P;
+    const int Hg = p.Hkv * p.P / HP;             // head groups per sequence: what one segment of visits serves
     const uint64_t block_bytes = p.block_bytes;
-    const uint64_t v_off = (uint64_t)p.Hkv * TILE;   // from a block's K tile to its V tile of the same head
+    const uint64_t v_off = (uint64_t)p.Hkv * TILE1;   // from a block's K tile to its V tile of the same head
     const int fused = (MODE == MODE_RESIDENT && p.k_new != nullptr) ? 1 : 0;
 
     // ---- this warp's contiguous share of the work.  Resident mode: the flat space of KV blocks
@@ -1287,7 +1284,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
                     const uint8_t *src = reinterpret_cast<const uint8_t *>(kv ? p.v_new : p.k_new) +
                                          ((size_t)s * p.Hkv + h) * (D * 2) + lane * 16;
                     uint8_t *dst =
-                        base + (size_t)(kv * p.Hkv + h) * TILE + (size_t)slot * (D * 2) + swz(lane, slot, row_vecs) * 16;
+                        base + (size_t)(kv * p.Hkv + h) * TILE1 + (size_t)slot * (D * 2) + swz(lane, slot, row_vecs) * 16;
                     *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
                 }
             } else if (lane == 0) {
@@ -1373,7 +1370,7 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
         if (cons_vis == 0) cons_phase ^= 1u;
 
         if (info & VF_NEW) {   // this step's token, attended to from the caller's rows
-            const int kvh = hg / p.P;
+            const int kvh = hg / p.P * HP;   // first KV head of the group
             mth.new_token(reinterpret_cast<const uint16_t *>(p.k_new) + ((size_t)s * p.Hkv + kvh) * D,
                           reinterpret_cast<const uint16_t *>(p.v_new) + ((size_t)s * p.Hkv + kvh) * D);
         }
@@ -1586,6 +1583,11 @@ __global__ void gather_kernel(const GatherParams p) {
 #define ISV_WARPS_GT1 16   // warps per CTA when one query head is handled per KV tile
 #endif
 
+#ifndef ISV_WARPS_PAIR80
+#define ISV_WARPS_PAIR80 12   // warps per CTA when a visit carries two KV heads at head_dim 80 (two heads' queries and
+                              // accumulators need more than the 128 registers that 16 warps leave a thread)
+#endif
+
 #ifndef ISV_WARPS_MMA
 #define ISV_WARPS_MMA 8   // warps per CTA of the tensor-core variant
 #endif
@@ -1597,16 +1599,23 @@ DecodeFn pick_mode(int mode) {
     return mode == MODE_RESIDENT ? decode_kernel<Math, MODE_RESIDENT, NW> : decode_kernel<Math, MODE_STAGED, NW>;
 }
 template <int D, bool BF16>
-DecodeFn pick_gt(int GT, int mode) {
+DecodeFn pick_gt(int GT, int HP, int mode) {
+    if (HP == 2) {   // multi-head attention, two adjacent KV heads per visit (small head dims only)
+        if constexpr (D < 128) {
+            if (GT == 2) return pick_mode<ScalarMath<D, 2, 16, BF16>, (D == 80 ? ISV_WARPS_PAIR80 : ISV_WARPS_GT1)>(mode);
+        }
+        return nullptr;
+    }
+    if (HP != 1) return nullptr;
     if (GT == 1) return pick_mode<ScalarMath<D, 1, 16, BF16>, ISV_WARPS_GT1>(mode);
     if (GT >= 2 && GT <= 16) return pick_mode<MmaMath<D, BF16>, (D == 64 ? 16 : D == 80 ? 12 : ISV_WARPS_MMA)>(mode);
     return nullptr;
 }
-DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
+DecodeFn pick(int D, int GT, int HP, int BT, bool bf16, int mode) {
     if (BT != 16) return nullptr;
-    if (D == 64) return bf16 ? pick_gt<64, true>(GT, mode) : pick_gt<64, false>(GT, mode);
-    if (D == 80) return bf16 ? pick_gt<80, true>(GT, mode) : pick_gt<80, false>(GT, mode);
-    if (D == 128) return bf16 ? pick_gt<128, true>(GT, mode) : pick_gt<128, false>(GT, mode);
+    if (D == 64) return bf16 ? pick_gt<64, true>(GT, HP, mode) : pick_gt<64, false>(GT, HP, mode);
+    if (D == 80) return bf16 ? pick_gt<80, true>(GT, HP, mode) : pick_gt<80, false>(GT, HP, mode);
+    if (D == 128) return bf16 ? pick_gt<128, true>(GT, HP, mode) : pick_gt<128, false>(GT, HP, mode);
     return nullptr;
 }
 
@@ -1615,35 +1624,38 @@ DecodeFn pick(int D, int GT, int BT, bool bf16, int mode) {
 // The tensor-core variant keeps 96 accumulator and operand registers per thread at head_dim 128 (8 warps),
 // 60 at head_dim 80 (12 warps fit without spills); at head_dim 64 it fits 128 registers, and 16 warps hide
 // its per-visit latencies (a visit carries only 4 KiB there).
-int decode_warps(int GT, int D) { return GT == 1 ? ISV_WARPS_GT1 : (D == 64 ? 16 : D == 80 ? 12 : ISV_WARPS_MMA); }
+int decode_warps(int GT, int D, int HP) {
+    if (HP == 2) return D == 80 ? ISV_WARPS_PAIR80 : ISV_WARPS_GT1;
+    return GT == 1 ? ISV_WARPS_GT1 : (D == 64 ? 16 : D == 80 ? 12 : ISV_WARPS_MMA);
+}
 
-int decode_default_stages(int D, int BT, int GT) {
-    const int per_stage = decode_warps(GT, D) * BT * D * 2;
+int decode_default_stages(int D, int BT, int GT, int HP) {
+    const int per_stage = decode_warps(GT, D, HP) * BT * D * 2 * HP;
     const int st = ((128 << 10) / per_stage) & ~1;   // slots come in pairs: a K and a V tile per block visit
     return st < 2 ? 2 : (st > 12 ? 12 : st);
 }
 
-size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode) {
-    const size_t tile = (size_t)BT * D * 2;
-    size_t b = (size_t)decode_warps(GT, D) * stages * (tile + 8 + 4 * V_WORDS);
+size_t decode_smem_bytes(int D, int BT, int GT, int HP, int stages, int max_seqs, int mode) {
+    const size_t tile = (size_t)BT * D * 2 * HP;
+    size_t b = (size_t)decode_warps(GT, D, HP) * stages * (tile + 8 + 4 * V_WORDS);
     if (mode == MODE_RESIDENT) b += (size_t)(2 * max_seqs + 1) * 4;
     return b;
 }
 
-cudaError_t decode_configure(int D, int GT, int BT, bool bf16, int mode, size_t smem) {
-    DecodeFn fn = pick(D, GT, BT, bf16, mode);
+cudaError_t decode_configure(int D, int GT, int HP, int BT, bool bf16, int mode, size_t smem) {
+    DecodeFn fn = pick(D, GT, HP, BT, bf16, mode);
     if (!fn) return cudaErrorInvalidValue;
     return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
-cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int BT, bool bf16, int mode, int grid,
+cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int HP, int BT, bool bf16, int mode, int grid,
                           int stages, size_t smem, cudaStream_t st) {
-    DecodeFn fn = pick(D, GT, BT, bf16, mode);
+    DecodeFn fn = pick(D, GT, HP, BT, bf16, mode);
     if (!fn || stages < 2) return cudaErrorInvalidValue;
     stages &= ~1;   // the kernel uses its ring slots in pairs
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(decode_warps(GT, D) * 32);
+    cfg.blockDim = dim3(decode_warps(GT, D, HP) * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

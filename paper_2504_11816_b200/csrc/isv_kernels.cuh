@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 namespace isv {
 
@@ -73,7 +74,8 @@ struct DecodeParams {
     float *acc_ml;              // [n_seqs][Hq][2]
     uint32_t *status;
     int32_t n_seqs, Hq, Hkv, P;
-    int32_t GT;                 // query heads of one head group (Hq = Hkv * P * GT)
+    int32_t GT;                 // query heads of one head group (Hq = Hkv * P * GT / HP, HP = KV heads per group:
+                                // fixed by the kernel variant, see pair_heads)
     int32_t finalize;           // resident: 1 = normalise and write out; 0 = leave (m, l, o) in acc_*
     int32_t early_reads;        // 1 = lengths, table and KV may be read before the dependency wait
     uint32_t spin_limit;        // polls after which a wait on a copy gives up (0 = default)
@@ -151,20 +153,30 @@ inline int group_heads(int G) {
     return 1;
 }
 
-// Warps per CTA of the decode kernel that handles GT query heads per KV tile at head_dim D.
-int decode_warps(int GT, int D);
+// KV heads whose tiles one block visit carries, for G query heads per KV head: 2 for multi-head attention
+// (G = 1) at head_dim 64 and 80 with an even head count - adjacent heads' tiles are contiguous in a block, one
+// copy brings both, and each is attended by its own query head, which halves the per-visit bookkeeping per
+// byte where tiles are small - else 1.  With 2, a head group is those two query heads (GT = 2).
+inline int pair_heads(int G, int D, int Hkv) {
+    if (const char *e = getenv("ISV_PAIR_HEADS"))   // tuning knob: 0 = one KV head per visit everywhere
+        if (atoi(e) == 0) return 1;
+    return (G == 1 && D < 128 && Hkv % 2 == 0) ? 2 : 1;
+}
+
+// Warps per CTA of the decode kernel that handles GT query heads per visit at head_dim D (HP: pair_heads).
+int decode_warps(int GT, int D, int HP);
 
 // Ring depth per warp (tile slots, an even number: a block visit takes a K and a V slot) that keeps about
 // 128 KiB of copies in flight per SM (measured on B200: deeper rings lower the achieved HBM rate).
-int decode_default_stages(int D, int BT, int GT);
+int decode_default_stages(int D, int BT, int GT, int HP);
 
 // Bytes of dynamic shared memory the decode kernel needs for `stages` ring
 // stages (one K or V tile each) per warp.
-size_t decode_smem_bytes(int D, int BT, int GT, int stages, int max_seqs, int mode);   // max_seqs: sequences x layers of a launch
+size_t decode_smem_bytes(int D, int BT, int GT, int HP, int stages, int max_seqs, int mode);   // max_seqs: sequences x layers of a launch
 
 // Launchers return the CUDA error of the launch.
-cudaError_t decode_configure(int D, int GT, int BT, bool bf16, int mode, size_t smem);
-cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int BT, bool bf16, int mode,
+cudaError_t decode_configure(int D, int GT, int HP, int BT, bool bf16, int mode, size_t smem);
+cudaError_t launch_decode(const DecodeParams &p, int D, int GT, int HP, int BT, bool bf16, int mode,
                           int grid, int stages, size_t smem, cudaStream_t st);
 cudaError_t launch_table_update(int32_t *table, const TableUpdateBatch &b, cudaStream_t st);
 cudaError_t launch_append(const AppendParams &p, cudaStream_t st);

@@ -83,8 +83,9 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     if (n_seqs == 0) return ISV_OK;
 
     const int G = q_heads / kv_heads;
-    const int GT = group_heads(G);
-    const int P = G / GT;
+    const int HP = pair_heads(G, head_dim, kv_heads);   // KV heads per head group
+    const int GT = HP == 2 ? 2 : group_heads(G);
+    const int P = HP == 2 ? 1 : G / GT;
     if ((long long)n_seqs * max_blocks_per_seq * kv_heads * P >= (1ll << 31))
         return err(ISV_EINVAL, "isv_attn_decode_static: n_seqs * blocks * heads too large");
 
@@ -119,8 +120,8 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     // A grid whose partials would not fit is cut down to the CTAs that do fit (the kernel is persistent
     // and divides the work among however many CTAs it gets); only a shape that leaves no room for one
     // CTA is refused.
-    const int nw = decode_warps(GT, head_dim);
-    const long long blocks = (long long)n_seqs * max_blocks_per_seq * kv_heads * P;
+    const int nw = decode_warps(GT, head_dim, HP);
+    const long long blocks = (long long)n_seqs * max_blocks_per_seq * kv_heads * P / HP;   // visits of the flat work list
     const int cap = max_ctas > 0 ? std::min(max_ctas, ds.sm_count) : ds.sm_count;
     int grid = (int)std::max<long long>(1, std::min<long long>(cap, (blocks + nw - 1) / nw));
     const size_t tickets_bytes = align256((size_t)n_seqs * kv_heads * P * 4);
@@ -142,13 +143,13 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     const bool bf16 = dtype == ISV_BF16;
     int stages = 0;
     size_t smem = 0;
-    for (int st = 2; st <= decode_default_stages(head_dim, block_tokens, GT); ++st) {
-        const size_t b = decode_smem_bytes(head_dim, block_tokens, GT, st, n_seqs, MODE_RESIDENT);
+    for (int st = 2; st <= decode_default_stages(head_dim, block_tokens, GT, HP); ++st) {
+        const size_t b = decode_smem_bytes(head_dim, block_tokens, GT, HP, st, n_seqs, MODE_RESIDENT);
         if (b <= (size_t)ds.smem_optin) { stages = st; smem = b; }
     }
     if (stages < 2) return err(ISV_EINVAL, "isv_attn_decode_static: shared memory too small for this shape");
     // the limit is raised to the device maximum so that it never undercuts another user of the kernel
-    e = decode_configure(head_dim, GT, block_tokens, bf16, MODE_RESIDENT, (size_t)ds.smem_optin);
+    e = decode_configure(head_dim, GT, HP, block_tokens, bf16, MODE_RESIDENT, (size_t)ds.smem_optin);
     if (e != cudaSuccess) return err(ISV_ECUDA, "isv_attn_decode_static: %s", cudaGetErrorString(e));
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -178,7 +179,7 @@ extern "C" int isv_attn_decode_static(const void *kv_pool_dev, int32_t n_pool_bl
     p.finalize = 1;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)head_dim));
     p.block_bytes = 2ull * kv_heads * block_tokens * head_dim * 2ull;
-    e = launch_decode(p, head_dim, GT, block_tokens, bf16, MODE_RESIDENT, grid, stages, smem, st);
+    e = launch_decode(p, head_dim, GT, HP, block_tokens, bf16, MODE_RESIDENT, grid, stages, smem, st);
     if (e != cudaSuccess) return err(ISV_ECUDA, "isv_attn_decode_static: %s", cudaGetErrorString(e));
     return ISV_OK;
 }

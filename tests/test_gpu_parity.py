@@ -101,9 +101,10 @@ def test_result_does_not_depend_on_split_or_chunk_size(ctas, chunk_blocks, q_hea
 
 # ---------------------------------------------------------------- head grouping, head dim, dtype
 
-# query heads per KV head: 1 runs on the CUDA cores, 2..16 as one tensor-core tile (2, 4, 8, 3, 16, 12, 5),
-# 32 as two passes of 16
-@pytest.mark.parametrize("q_heads,kv_heads", [(8, 8), (8, 4), (8, 2), (16, 2), (6, 2), (32, 2), (24, 2), (10, 2),
+# query heads per KV head: 1 runs on the CUDA cores (at head_dim 64 / 80 two adjacent KV heads per visit when the
+# head count is even: 8 heads; one per visit otherwise: 5 heads), 2..16 as one tensor-core tile (2, 4, 8, 3, 16,
+# 12, 5), 32 as two passes of 16
+@pytest.mark.parametrize("q_heads,kv_heads", [(8, 8), (5, 5), (8, 4), (8, 2), (16, 2), (6, 2), (32, 2), (24, 2), (10, 2),
                                               (64, 2)])
 @pytest.mark.parametrize("head_dim", [64, 80, 128])
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
