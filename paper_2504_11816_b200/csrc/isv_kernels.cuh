@@ -19,8 +19,9 @@ enum DecodeMode : int { MODE_RESIDENT = 0, MODE_STAGED = 1 };
 //     host-flagged newest block from its tail slot, skips other host blocks.
 //     A (sequence, head group) that spans several warps is finished by
 //     whichever of them arrives last (ticket), which merges their partials.
-//   A head group is GT query heads that share a KV head and are handled together on one KV tile:
-//     GT = 1 on the CUDA cores, 2..16 on the tensor cores (group_heads picks it).
+//   A head group is the GT query heads one block visit serves: GT = 2..16 query heads that share a KV head,
+//     on the tensor cores (group_heads picks GT); or, for multi-head attention, on the CUDA cores, one query
+//     head with its KV head (GT = 1) or two adjacent ones, each with its own KV head (GT = 2, pair_heads).
 //   MODE_STAGED: units are (chunk unit, kv head x pass) from the plan lists;
 //     blocks are read from the staging buffer; results are merged into the
 //     running state acc_o / acc_ml, which one unit per launch owns.
