@@ -11,7 +11,7 @@ The default workload is the offload sweep the metric is named after: the
 13B-shaped ragged batch (c5) at offload fractions 0 / 0.25 / 0.5 / 0.75 / 1, the
 7B-shaped batches with nothing (c2) and half (c3) of the cache offloaded, the
 8B-GQA batch with three quarters (c4) and nothing offloaded, and the paper's
-own OPT-2.7B offline shape.  The headline figures (`value`, `config`, `roofline`, `e2e`) are
+own OPT-2.7B offline shape at its Table VI offload ratios (0 / 0.6 / 1).  The headline figures (`value`, `config`, `roofline`, `e2e`) are
 those of c5 at offload fraction 0.5, timed for exactly --steps steps after
 --warmup warm-up steps; every other point is listed under `sweep` with its own
 step counts, its tokens/s, its fraction of the combined HBM / host-link
@@ -181,6 +181,8 @@ def sweep_points(K, Wm, layers=None, batch=None):
     C = W.CONFIGS
     pts = [(C["c2"], 120, max(3, min(Wm, 8)), 3, True),
            (C["opt2.7b"], 120, max(3, min(Wm, 8)), 3, True),
+           (C["opt2.7b"].with_(offload_frac=0.6), 4, 3, 1, False),    # the offload ratios of the paper's Table VI
+           (C["opt2.7b"].with_(offload_frac=1.0), 4, 3, 1, False),
            (C["c3"], 4, 3, 1, False),
            (C["c4"], 4, 3, 1, False),
            (C["c4"].with_(offload_frac=0.0), 9, 3, 3, False),     # the grouped-query (tensor-core) variant at the HBM rate

@@ -80,7 +80,7 @@ def test_default_run_is_the_offload_sweep():
     d = _run("--batch", "4", "--layers", "2", "--steps", "3", "--warmup", "3", "--no-cpu-baseline")
     assert d["config"]["workload"].startswith("c5:") and d["config"]["offload_frac"] == 0.5
     pts = {(p["name"], p["offload_frac"]) for p in d["sweep"]}
-    assert pts == {("c2", 0.0), ("opt2.7b", 0.0), ("c3", 0.5), ("c4", 0.75), ("c4", 0.0)} | \
+    assert pts == {("c2", 0.0), ("opt2.7b", 0.0), ("opt2.7b", 0.6), ("opt2.7b", 1.0), ("c3", 0.5), ("c4", 0.75), ("c4", 0.0)} | \
         {("c5", f) for f in (0.0, 0.25, 0.5, 0.75, 1.0)}
     for p in d["sweep"]:
         assert p["tokens_per_s"] > 0 and p["combined_roofline_frac"] > 0 and p["device_status"] == 0
