@@ -917,6 +917,7 @@ static int decode_impl(isv_kv *h, int32_t layer, const void *q, void *out, float
         if (k_new) {
             p.k_new = k_new; p.v_new = v_new;
             p.lens_out = lens_ptr(h, layer, 1);
+            p.lens_count = g.max_seqs;
             p.pool_w = h->pool_hbm + slab_hbm(h, layer);
             p.tail_w = h->tail ? h->tail + slab_tail(h, layer) : nullptr;
             // the kernel launched just before this one (the previous layer's, or a caller's) writes neither
@@ -1085,6 +1086,7 @@ static int decode_layers_fused(isv_kv *h, int l0, int nl, const void *q, const v
     p.finalize = split ? 0 : 1;
     p.n_layers = nl; p.layer0 = l0; p.phys_layers = g.phys_layers;
     p.lens = h->lens_dev; p.lens_out = h->lens_dev;
+    p.lens_count = g.max_seqs;
     p.lens_layer_stride = g.max_seqs;
     p.lens_copy_stride = g.layers * g.max_seqs;
     for (int l = 0; l < g.layers; ++l)

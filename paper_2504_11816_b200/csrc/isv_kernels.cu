@@ -1292,6 +1292,22 @@ __global__ void __launch_bounds__(NW * 32, 1) decode_kernel(const DecodeParams p
             }
             if (kv == 0 && h == 0 && lane == 0) lens_out[row] = len + 1;
         }
+        // sequences beyond those of this launch keep their lengths: carry them over to the copy that becomes
+        // current, so that a later launch over more sequences finds them
+        if (p.lens_count > NSEQ) {
+            const int extra = p.lens_count - NSEQ;
+            for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < NL * extra; i += gridDim.x * blockDim.x) {
+                const int l = i / extra, sx = NSEQ + (i - l * extra);
+                if (NL > 1) {
+                    const int la = p.layer0 + l;
+                    const size_t cur = (size_t)((p.lens_cur_mask >> la) & 1);
+                    const size_t at = (size_t)la * p.lens_layer_stride + sx;
+                    p.lens_out[(cur ^ 1) * p.lens_copy_stride + at] = p.lens[cur * p.lens_copy_stride + at];
+                } else {
+                    p.lens_out[sx] = p.lens[sx];
+                }
+            }
+        }
     }
 
     // Publishes a stored partial: fence, ticket, and the merge if this was the last split to arrive.

@@ -45,7 +45,9 @@ struct DecodeParams {
     // this step's token; the kernel stores the token's K/V rows into the cache, writes lens + 1 to
     // lens_out, and attends to the new token straight from k_new / v_new
     const void *k_new, *v_new;  // [n_seqs][Hkv][D] 16-bit, or NULL
-    int32_t *lens_out;          // [n_seqs]
+    int32_t *lens_out;          // [lens_count]
+    int32_t lens_count;         // entries of `lens` / `lens_out` per layer (>= n_seqs): those beyond n_seqs are
+                                // copied over unchanged
     uint8_t *pool_w, *tail_w;   // writable aliases of pool / tail
     // several layers in one launch (resident mode with fused append only): n_layers > 1 makes the launch
     // cover logical layers layer0 .. layer0 + n_layers - 1 of one decode step.  The work list is then the

@@ -487,6 +487,38 @@ def test_host_buffer_step_equals_device_buffer_step(f, phys):
         hb.check_gather(layers=range(layers - phys, layers))
 
 
+@pytest.mark.parametrize("f", [0.0, 0.5])
+def test_step_call_over_the_first_sequences_only(f):
+    """isv_decode_step with n_seqs below the cache's capacity: only those sequences advance (in every layer), the
+    arrays hold n_seqs rows per layer, and the others keep their lengths and content; a later step advances all."""
+    lens = [90, 16, 47, 200, 5]
+    layers, n = 3, 3
+    w = small(batch=len(lens), steps=6, f=f, perm=23, ctx=(5, 200), layers=layers, q_heads=8, kv_heads=8, head_dim=64,
+              seed=41)
+    with Harness(w, lens=lens) as hz:
+        hz.fill()
+        for t in range(4):
+            m = n if t < 3 else w.batch                      # three partial steps, then a full one
+            ks, vs, qs = zip(*[W.host_step(w, hz.rng) for _ in range(layers)])
+            k, v, q = (np.stack(x)[:, :m] for x in (ks, vs, qs))
+            kd, vd, qd = (bits_to_dev(np.ascontiguousarray(x), w.dtype) for x in (k, v, q))
+            of = torch.full((layers, m, w.q_heads, w.head_dim), float("nan"), device="cuda")
+            torch.cuda.synchronize()
+            B.isv_decode_step(hz.h, qd, kd, vd, None, of, m)
+            assert B.isv_sync(hz.h) == 0
+            o = of.cpu().numpy()
+            for layer in range(layers):
+                hz.shadow.append(layer, np.ascontiguousarray(k[layer]), np.ascontiguousarray(v[layer]))
+                full_q = np.zeros((w.batch, w.q_heads, w.head_dim), np.uint16)
+                full_q[:m] = q[layer]
+                ref = hz.reference(layer, full_q, seqs=range(m))
+                assert np.max(np.abs(o[layer] - ref)) <= TOL
+            hz.cur[:m] += 1
+            for layer in range(layers):
+                assert np.array_equal(B.isv_seq_lens_host(hz.h, layer, w.batch), hz.cur)
+        hz.check_gather()
+
+
 def test_device_lengths_beyond_the_table_row_are_clamped_and_flagged():
     """Caller-supplied device lengths are not trusted: one that exceeds what a table row covers (or is
     negative) is clamped, the status word says so, and the other sequences are unaffected."""
