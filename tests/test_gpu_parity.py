@@ -519,6 +519,45 @@ def test_step_call_over_the_first_sequences_only(f):
         hz.check_gather()
 
 
+@pytest.mark.parametrize("f", [0.0, 0.5])
+def test_a_full_sequence_refuses_the_step_and_changes_nothing(f):
+    """When a sequence has reached max_tokens_per_seq the step is refused with ISV_ECAPACITY before anything is
+    enqueued: no layer's lengths move, the cache still reads back bit for bit, and attention over it still works."""
+    lens = [30, 47, 48]
+    layers = 3
+    w = small(batch=len(lens), steps=2, f=f, perm=29, ctx=(30, 48), layers=layers, q_heads=4, kv_heads=4, head_dim=128,
+              seed=43)
+    with Harness(w, lens=lens) as hz:                    # capacity 48 + 2 = 50 tokens
+        hz.fill()
+        for t in range(2):
+            hz.check_step(hz.step(fused=True))
+        assert int(hz.cur.max()) == 50
+        ks, vs, qs = zip(*[W.host_step(w, hz.rng) for _ in range(layers)])
+        k, v, q = (np.stack(x) for x in (ks, vs, qs))
+        kd, vd, qd = (bits_to_dev(x, w.dtype) for x in (k, v, q))
+        of = torch.zeros((layers, w.batch, w.q_heads, w.head_dim), device="cuda")
+        torch.cuda.synchronize()
+        with pytest.raises(B.IsvError) as ei:
+            B.isv_decode_step(hz.h, qd, kd, vd, None, of, w.batch)
+        assert ei.value.code == B.ISV_ECAPACITY and "full" in ei.value.message
+        assert B.isv_sync(hz.h) == 0
+        for layer in range(layers):
+            assert np.array_equal(B.isv_seq_lens_host(hz.h, layer, w.batch), hz.cur)
+        hz.check_gather()
+        # the first two sequences still have room: a step over them alone goes through
+        of2 = torch.full((layers, 2, w.q_heads, w.head_dim), float("nan"), device="cuda")
+        k2, v2, q2 = (np.ascontiguousarray(x[:, :2]) for x in (k, v, q))
+        B.isv_decode_step(hz.h, bits_to_dev(q2, w.dtype), bits_to_dev(k2, w.dtype), bits_to_dev(v2, w.dtype), None, of2, 2)
+        assert B.isv_sync(hz.h) == 0
+        for layer in range(layers):
+            hz.shadow.append(layer, k2[layer], v2[layer])
+            full_q = np.zeros((w.batch, w.q_heads, w.head_dim), np.uint16)
+            full_q[:2] = q2[layer]
+            assert np.max(np.abs(of2[layer].cpu().numpy() - hz.reference(layer, full_q, seqs=range(2)))) <= TOL
+        hz.cur[:2] += 1
+        hz.check_gather()
+
+
 def test_device_lengths_beyond_the_table_row_are_clamped_and_flagged():
     """Caller-supplied device lengths are not trusted: one that exceeds what a table row covers (or is
     negative) is clamped, the status word says so, and the other sequences are unaffected."""
