@@ -47,14 +47,14 @@ HEADLINE = ("c5", 0.5)
 
 # DRAM traffic of the resident decode kernel from one ncu capture (bytes per KV byte
 # processed), valid only for the kernel source it was taken from.
-NCU_TRAFFIC = {"kernels_sha1": "0fa378a9390c00115aca2be545f1133c02540fed",
-               # multi-head shapes (CUDA-core arithmetic): (1094.10 MB read + 5.67 MB written) / 1078.46 MB
+NCU_TRAFFIC = {"kernels_sha1": "44aed6d32aaf25000f3eb95c035535f0ed28b65a",
+               # multi-head shapes (CUDA-core arithmetic): (1094.13 MB read + 5.94 MB written) / 1078.46 MB
                # algorithmic, 2-layer case of the 7B shape (one launch per step)
-               "dram_bytes_per_kv_byte": (1094.096 + 5.671) / 1078.460416,
+               "dram_bytes_per_kv_byte": (1094.131 + 5.939) / 1078.460416,
                "source": "profiles/decode_kernel_c2_2layers.md",
-               # grouped-query shapes (tensor-core arithmetic): (1080.08 MB + 5.44 MB) / 1074.92 MB, 32 sequences
+               # grouped-query shapes (tensor-core arithmetic): (1080.11 MB + 5.11 MB) / 1074.92 MB, 32 sequences
                # and 2 layers of the 8B-GQA shape
-               "dram_bytes_per_kv_byte_gqa": (1080.079 + 5.439) / 1074.921472,
+               "dram_bytes_per_kv_byte_gqa": (1080.107 + 5.109) / 1074.921472,
                "source_gqa": "profiles/decode_kernel_gqa_c4shape_batch32_2layers.md"}
 
 

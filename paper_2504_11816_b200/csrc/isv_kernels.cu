@@ -532,6 +532,11 @@ struct MmaMath {
     uint32_t ph[4], pl[4];      // weights of the current block as A fragments: 16-bit value and remainder
     float scale;
     int lane, r, c, gt;
+    // Byte offsets, inside a tile, of the rows this lane addresses in the matrix loads.  A load of 16-dim step
+    // ks wants 16-byte chunk 2 ks + h of token row t (h: the lane's half of the step); with the stored chunk
+    // order that is chunk position 8 (ks / 4) + ((2 (ks % 4) + h) ^ (t % 8)): four lane-dependent values per
+    // operand, plus 128 bytes per group of eight chunks, which goes into the instruction as an immediate.
+    uint32_t koff[4], voff[4];
 
     __device__ __forceinline__ void init(const DecodeParams &p, int lane_) {
         lane = lane_;
@@ -539,6 +544,19 @@ struct MmaMath {
         c = lane_ & 3;
         gt = p.GT;
         scale = p.scale_log2;
+        const int t7 = lane_ & 7;
+        const int ktok = ((lane_ >> 4) << 3) + t7, khalf = (lane_ >> 3) & 1;   // K: plain loads
+        const int vtok = (((lane_ >> 3) & 1) << 3) + t7, vhi = lane_ >> 4;     // V: transposing loads
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            koff[j] = ktok * ROW + ((((2 * j + khalf) ^ t7) & 7) << 4);
+            voff[j] = vtok * ROW + ((((2 * j + vhi) ^ t7) & 7) << 4);
+        }
+    }
+    // Offset of step ks for an operand whose four lane-dependent offsets are off[]: steps inside the complete
+    // groups of eight chunks are permuted, a trailing incomplete group (head_dim 80: chunks 8 and 9) is not.
+    __device__ __forceinline__ uint32_t step_off(const uint32_t (&off)[4], int ks, int tok_row_bytes, int h) const {
+        return (2 * ks < ((D / 8) & ~7)) ? off[ks & 3] + 128 * (ks >> 2) : tok_row_bytes + ((2 * ks + h) << 4);
     }
     __device__ __forceinline__ int heads() const { return gt; }
 
@@ -578,13 +596,12 @@ struct MmaMath {
 
     __device__ __forceinline__ void k_tile(const uint8_t *tile, int ntok) {
         float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};   // tokens 0..7 and 8..15
-        const int tok = ((lane >> 4) << 3) + (lane & 7);
-        const uint32_t rowaddr = smem_u32(tile) + tok * ROW;
-        const int half = (lane >> 3) & 1;
+        const uint32_t base = smem_u32(tile);
+        const int tok = ((lane >> 4) << 3) + (lane & 7), half = (lane >> 3) & 1;   // (used by the unpermuted tail only)
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
             uint32_t b0, b1, b2, b3;
-            ldsm_x4(rowaddr + (swz(2 * ks + half, tok, D / 8) << 4), b0, b1, b2, b3);
+            ldsm_x4(base + step_off(koff, ks, tok * ROW, half), b0, b1, b2, b3);
             mma16816<BF16>(s0, qa[ks], b0, b1);
             mma16816<BF16>(s1, qa[ks], b2, b3);
         }
@@ -625,9 +642,8 @@ struct MmaMath {
     }
 
     __device__ __forceinline__ void v_tile(const uint8_t *tile, int ntok) {
-        const int tok = (((lane >> 3) & 1) << 3) + (lane & 7);
-        const uint32_t rowaddr = smem_u32(tile) + tok * ROW;
-        const int hi = lane >> 4;
+        const uint32_t base = smem_u32(tile);
+        const int tok = (((lane >> 3) & 1) << 3) + (lane & 7), hi = lane >> 4;     // (used by the unpermuted tail only)
         uint32_t k0 = 0xffffffffu, k1 = 0xffffffffu;   // keep-masks of the token pairs (2c, 2c+1) and (2c+8, 2c+9)
         if (ntok < BT) {
             k0 = (2 * c < ntok ? 0x0000ffffu : 0u) | (2 * c + 1 < ntok ? 0xffff0000u : 0u);
@@ -636,7 +652,7 @@ struct MmaMath {
 #pragma unroll
         for (int jp = 0; jp < D / 16; ++jp) {
             uint32_t b0, b1, b2, b3;
-            ldsm_x4_t(rowaddr + (swz(2 * jp + hi, tok, D / 8) << 4), b0, b1, b2, b3);
+            ldsm_x4_t(base + step_off(voff, jp, tok * ROW, hi), b0, b1, b2, b3);
             if (ntok < BT) {   // never let unspecified bits (possibly NaN patterns) reach a product
                 b0 &= k0; b1 &= k1; b2 &= k0; b3 &= k1;
             }
