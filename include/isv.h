@@ -336,8 +336,10 @@ int isv_link_probe(uint64_t bytes, int32_t reps, double *h2d_gbs, double *d2h_gb
  *          must stay valid and unchanged while the handle lives
  *   x_dev  [M][K] 16-bit;  y_dev [M][N] 16-bit and / or y_f32_dev [M][N] fp32 (one may be NULL)
  * isv_linear_create allocates split-K scratch and encodes the weight's tensor map (synchronous);
- * isv_linear_forward enqueues one kernel on `stream` (asynchronous); isv_linear_status waits for
- * the stream and returns ISV_EDEVICE_STATUS if a bounded wait inside the kernel expired. */
+ * isv_linear_forward enqueues the streaming kernel and, where tiles of the output are shared by
+ * several CTAs, a small kernel that adds their partial sums, on `stream` (asynchronous, no host
+ * wait); isv_linear_status waits for the stream and returns ISV_EDEVICE_STATUS if a bounded wait
+ * inside the kernel expired. */
 typedef struct isv_linear isv_linear;
 int isv_linear_create(isv_linear **out, const void *w_dev, int32_t N, int32_t K, int32_t dtype,
                       int32_t max_M, void *stream);

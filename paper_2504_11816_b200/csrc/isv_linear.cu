@@ -11,8 +11,10 @@
 //     (kind::f16, fp32 accumulation in tensor memory) and releases ring stages with
 //     tcgen05.commit; four epilogue warps read the accumulator with tcgen05.ld;
 //   - the (column tile, K block) list is cut into equal ranges, one per persistent CTA, so every
-//     SM streams the same number of weight bytes; a tile shared by several CTAs is summed from
-//     their fp32 partials, in fixed order, by the last of them to arrive.
+//     SM streams the same number of weight bytes; a CTA leaves the fp32 partial of a tile it shares
+//     with others in global memory and exits, and a second, small kernel adds a tile's partials in
+//     fixed order.  The streaming CTAs thus all end together and free their shared memory at once,
+//     so the next call's CTAs can fill their rings with weights while the sums are still being taken.
 // Every wait is bounded; on expiry the kernel flags the status word, still frees its tensor
 // memory and returns.
 #include <cuda.h>
@@ -136,11 +138,11 @@ struct LinearParams {
     void *y;                 // [M][N] 16-bit or NULL
     float *y_f32;            // [M][N] or NULL
     float *partials;         // [2 * grid][M][128] fp32: a CTA leaves at most two partial tiles
-    int32_t *tickets;        // [N / 128], zero between launches
     uint32_t *status;
     int32_t M, N, K;
     int32_t mma_n;           // batch padded to a multiple of 16
     int32_t stages, tmem_cols, bf16;
+    int32_t grid_main;       // CTAs of linear_kernel (the reduction needs the same cut)
 };
 
 __device__ __forceinline__ void store_out(const LinearParams &p, int m, int n, float v) {
@@ -181,14 +183,21 @@ __device__ __forceinline__ void store_out4(const LinearParams &p, int m, int n, 
 // contiguous ranges, one per CTA (persistent, one CTA per SM), so every SM streams the same number
 // of weight bytes whatever the matrix shape.  A run of K blocks of one tile inside a range is a
 // segment: a segment that covers its whole tile is stored directly, otherwise its fp32 partial goes
-// to one of the CTA's two slots and the last CTA of that tile to arrive adds the partials in fixed
-// order.  The ring of TMA stages runs across segments without draining, and two accumulators in
-// tensor memory let the epilogue of one segment overlap the MMAs of the next.
+// to one of the CTA's two slots (slot 0 if the segment opens the CTA's range, else slot 1) and
+// linear_reduce_kernel adds the partials in fixed order.  The ring of TMA stages runs across
+// segments without draining, and two accumulators in tensor memory let the epilogue of one segment
+// overlap the MMAs of the next.
 struct Cut {
     long long total;
     int n;
     __device__ long long first(int c) const { return total * c / n; }
     __device__ int range_of(long long x) const { return (int)(((x + 1) * n - 1) / total); }
+    __device__ static Cut of(const LinearParams &p, int grid) {
+        Cut c;
+        c.total = (long long)(p.N / kTileN) * (p.K / kTileK);
+        c.n = (int)min((long long)grid, c.total);
+        return c;
+    }
 };
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -198,9 +207,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     uint8_t *smem = smem_raw + ((1024u - (s32(smem_raw) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kblocks = p.K / kTileK;
-    Cut cut;
-    cut.total = (long long)(p.N / kTileN) * kblocks;
-    cut.n = (int)min((long long)gridDim.x, cut.total);
+    const Cut cut = Cut::of(p, gridDim.x);
     const int cta = blockIdx.x;
     if (cta >= cut.n) return;
     const long long f0 = cut.first(cta), f1 = cut.first(cta + 1);
@@ -215,8 +222,8 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     uint64_t *acc_empty = acc_full + 2;         // [2]
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
     volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    volatile int *is_last = failed + 1;
-    volatile int *ep_fail = failed + 2;   // written and read by the epilogue warps only, around their barrier
+    volatile int *ep_fail = failed + 1;   // written and read by the epilogue warps only, around their barrier
+    const int prefill = (int)min((long long)p.stages, f1 - f0);
 
     if (threadIdx.x == 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
@@ -235,6 +242,17 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         *ep_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // The weights never change, so the ring is filled with weight tiles at once, before tensor memory
+        // is allocated and before the kernels launched ahead of this one have finished (programmatic
+        // dependent launch): the ramp-up overlaps the previous kernel's tail.  The matching activation
+        // tiles follow once that kernel is complete.
+        for (int it = 0; it < prefill; ++it) {
+            const long long f = f0 + it;
+            const uint32_t bar = s32(&full[it]);
+            mbar_expect_tx(bar, a_bytes + b_bytes);
+            tma_load_3d(s32(ring + (size_t)it * stage_bytes), &map_w, (int)(f / kblocks) * kTileN,
+                        (int)(f % kblocks) * kSub, bar);
+        }
     }
     if (warp == 1) {   // tensor memory: two accumulators of mma_n columns, power-of-two total
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(tmem_slot)), "r"(p.tmem_cols)
@@ -250,17 +268,6 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     if (warp == 0) {
         // ---- producer: one thread walks the CTA's range and issues the TMA copies
         if (lane == 0) {
-            // The weights never change, so the ring is first filled with weight tiles; only then does the
-            // producer wait for the kernels launched before this one (programmatic dependent launch) and
-            // fetch the matching activation tiles.  The ramp-up thus overlaps the previous kernel's tail.
-            const int prefill = (int)min((long long)p.stages, f1 - f0);
-            for (int it = 0; it < prefill; ++it) {
-                const long long f = f0 + it;
-                const uint32_t bar = s32(&full[it]);
-                mbar_expect_tx(bar, a_bytes + b_bytes);
-                tma_load_3d(s32(ring + (size_t)it * stage_bytes), &map_w, (int)(f / kblocks) * kTileN,
-                            (int)(f % kblocks) * kSub, bar);
-            }
             asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int it = 0; it < prefill; ++it)
                 tma_load_3d(s32(ring + (size_t)it * stage_bytes + a_bytes), &map_x, 0,
@@ -320,8 +327,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
         // ---- epilogue: warp w reads tensor-memory lanes [32 * (w % 4), +32) = weight rows of the tile
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
-        const int et = threadIdx.x - 64;              // 0..127 among the epilogue threads
-        asm volatile("griddepcontrol.wait;" ::: "memory");   // outputs, partials and tickets may still be in use
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // outputs and partials may still be in use
         int g = 0;
         for (long long f = f0; f < f1; ++g) {
             const int t = (int)(f / kblocks);
@@ -357,55 +363,6 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(&acc_empty[b])) : "memory");
-            if (complete) continue;
-            // ---- partial tile: publish, and combine if every contributor of the tile has arrived
-            const int cf = cut.range_of(start), cl = cut.range_of(start + kblocks - 1);
-            const int nc = cl - cf + 1;
-            __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");          // the four epilogue warps
-            if (et == 0) {
-                const int ticket = atomicAdd(&p.tickets[t], 1);
-                *is_last = (ticket == nc - 1);
-                if (*is_last) p.tickets[t] = 0;
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (*is_last) {
-                __threadfence();
-                const int cf_slot = (cut.first(cf) == start) ? 0 : 1;
-                // Thread (cg, mg) sums 4 adjacent columns of every 4th token, 8 tokens per round, from all
-                // contributors in their fixed order; a warp's load covers one whole 512-byte row of a partial,
-                // and the loads of a round (two contributors at a time) are in flight together.
-                const int cg = et & 31, mg = et >> 5;
-                constexpr int MB = 8;
-                const int n0 = t * kTileN + 4 * cg;
-                for (int mb = mg; mb < p.M; mb += 4 * MB) {
-                    float4 acc[MB];
-#pragma unroll
-                    for (int j = 0; j < MB; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 2
-                    for (int c = 0; c < nc; ++c) {
-                        const int sl = c == 0 ? 2 * cf + cf_slot : 2 * (cf + c);
-                        const float *src = p.partials + (size_t)sl * p.M * kTileN + 4 * cg;
-                        float4 v[MB];
-#pragma unroll
-                        for (int j = 0; j < MB; ++j) {
-                            const int m = mb + 4 * j;
-                            v[j] = m < p.M ? __ldcg(reinterpret_cast<const float4 *>(src + (size_t)m * kTileN))
-                                           : make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-#pragma unroll
-                        for (int j = 0; j < MB; ++j) {
-                            acc[j].x += v[j].x; acc[j].y += v[j].y; acc[j].z += v[j].z; acc[j].w += v[j].w;
-                        }
-                    }
-#pragma unroll
-                    for (int j = 0; j < MB; ++j) {
-                        const int m = mb + 4 * j;
-                        if (m < p.M) store_out4(p, m, n0, acc[j]);
-                    }
-                }
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");          // is_last is reused by the next partial
         }
     }
 
@@ -415,6 +372,68 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
     }
+}
+
+// Adds the partials of every tile that several CTAs of linear_kernel shared: CTA (tile, group of
+// kRedRows tokens), thread = 4 adjacent outputs of one token, contributors in their fixed order, kFly
+// of them in flight at a time.  Its loads queue behind the weight tiles that the next call's CTAs are
+// already fetching, so a round trip costs 1.5-2 us: a small grid takes up to eight contributors in
+// one round; a large grid (many tokens) keeps four, because more registers per thread would leave too
+// few of these CTAs beside the streaming ones (measured slower).  It runs as a programmatic dependent
+// of linear_kernel; every CTA waits for that kernel, also one with nothing to add, so that this grid
+// never completes first.
+constexpr int kRedThreads = 256, kRedRows = 2 * (kRedThreads / 32);
+
+// 16-byte load that bypasses L1, issued only if `pred`; the result is zero otherwise
+__device__ __forceinline__ float4 ldcg_if(const float *src, bool pred) {
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    asm volatile(
+        "{\n.reg .pred q;\nsetp.ne.b32 q, %5, 0;\n@q ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];\n}\n"
+        : "+f"(v.x), "+f"(v.y), "+f"(v.z), "+f"(v.w)
+        : "l"(src), "r"((int)pred)
+        : "memory");
+    return v;
+}
+
+template <int kFly>
+__global__ void __launch_bounds__(kRedThreads, kFly == 4 ? 4 : 2) linear_reduce_kernel(const LinearParams p) {
+    const int kblocks = p.K / kTileK;
+    const Cut cut = Cut::of(p, p.grid_main);
+    const int groups = (p.M + kRedRows - 1) / kRedRows;
+    const int t = blockIdx.x / groups, m0 = (blockIdx.x % groups) * kRedRows;
+    const long long start = (long long)t * kblocks;
+    const int cf = cut.range_of(start), cl = cut.range_of(start + kblocks - 1);
+    const int nc = cl - cf + 1;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (nc == 1) return;                              // the tile was stored whole by its one CTA
+    if (m0 + (int)(threadIdx.x >> 5) >= p.M) return;  // this warp's tokens lie beyond the batch
+    const int cf_slot = (cut.first(cf) == start) ? 0 : 1;
+    const int cg = threadIdx.x & 31, mr = threadIdx.x >> 5;
+    const int m[2] = {m0 + mr, m0 + mr + kRedThreads / 32};
+    float4 acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+    for (int c0 = 0; c0 < nc; c0 += kFly) {
+        float4 v[kFly][2];
+#pragma unroll
+        for (int j = 0; j < kFly; ++j) {
+            // predicated loads, not branches, so that all of them are issued before the first is used
+            const int c = min(c0 + j, nc - 1);
+            const int sl = c == 0 ? 2 * cf + cf_slot : 2 * (cf + c);
+            const float *src = p.partials + (size_t)sl * p.M * kTileN + 4 * cg;
+#pragma unroll
+            for (int r = 0; r < 2; ++r)
+                v[j][r] = ldcg_if(src + (size_t)min(m[r], p.M - 1) * kTileN, c0 + j < nc && m[r] < p.M);
+        }
+#pragma unroll
+        for (int j = 0; j < kFly; ++j)
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {   // adding the zeros of a load that was not issued changes nothing
+                acc[r].x += v[j][r].x; acc[r].y += v[j][r].y; acc[r].z += v[j][r].z; acc[r].w += v[j][r].w;
+            }
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r)
+        if (m[r] < p.M) store_out4(p, m[r], t * kTileN + 4 * cg, acc[r]);
 }
 
 // ---------------------------------------------------------------- host side
@@ -462,7 +481,7 @@ struct isv_linear {
     CUtensorMap map_w;
     int grid = 1;
     float *partials = nullptr;
-    int32_t *tickets = nullptr;
+    bool split = false;   // some tile is shared by several CTAs: the reduction kernel follows every launch
     uint32_t *status = nullptr;
     int smem_optin = 0;
 };
@@ -473,7 +492,6 @@ int isv_linear_free(isv_linear *l) {
     if (!l) return err(ISV_EINVAL, "null handle");
     if (l->stream) cudaStreamSynchronize(l->stream);
     cudaFree(l->partials);
-    cudaFree(l->tickets);
     cudaFree(l->status);
     delete l;
     return ISV_OK;
@@ -501,9 +519,12 @@ int isv_linear_create(isv_linear **out, const void *w_dev, int32_t N, int32_t K,
     l->grid = sms;                      // persistent: one CTA per SM (two per SM with half the ring each measured no faster)
     int rc = make_map(&l->map_w, w_dev, N, K, kTileN, l->bf16);
     if (rc) { delete l; return rc; }
-    e = cudaMalloc((void **)&l->tickets, (size_t)n_tiles * 4);
-    if (e == cudaSuccess) e = cudaMemset(l->tickets, 0, (size_t)n_tiles * 4);
-    if (e == cudaSuccess) e = cudaMalloc((void **)&l->status, 4);
+    {   // the kernel's cut of the (tile, K block) list: a range border inside a tile splits that tile
+        const long long kblocks = K / kTileK, total = (long long)n_tiles * kblocks;
+        const long long n = std::min<long long>(l->grid, total);
+        for (long long c = 1; c < n && !l->split; ++c) l->split = (total * c / n) % kblocks != 0;
+    }
+    e = cudaMalloc((void **)&l->status, 4);
     if (e == cudaSuccess) e = cudaMemset(l->status, 0, 4);
     if (e == cudaSuccess) e = cudaMalloc((void **)&l->partials, (size_t)2 * l->grid * max_M * kTileN * 4);
     // the kernel also has a few bytes of static shared memory: leave room for them under the limit
@@ -524,10 +545,11 @@ int isv_linear_forward(isv_linear *l, const void *x_dev, void *y_dev, float *y_f
     if ((reinterpret_cast<uintptr_t>(x_dev) & 15u)) return err(ISV_EINVAL, "x must be 16-byte aligned");
     if (M < 1 || M > l->max_M) return err(ISV_EINVAL, "M (%d) must be in [1, %d]", M, l->max_M);
     LinearParams p{};
-    p.y = y_dev; p.y_f32 = y_f32_dev; p.partials = l->partials; p.tickets = l->tickets; p.status = l->status;
+    p.y = y_dev; p.y_f32 = y_f32_dev; p.partials = l->partials; p.status = l->status;
     p.M = M; p.N = l->N; p.K = l->K;
     p.mma_n = std::max(16, (M + 15) / 16 * 16);
     p.bf16 = l->bf16 ? 1 : 0;
+    p.grid_main = l->grid;
     int cols = 32;
     while (cols < 2 * p.mma_n) cols *= 2;        // two accumulators
     p.tmem_cols = cols;
@@ -556,6 +578,14 @@ int isv_linear_forward(isv_linear *l, const void *x_dev, void *y_dev, float *y_f
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, linear_kernel, l->map_w, map_x, p);
+    if (e == cudaSuccess && l->split) {
+        const int red_grid = (l->N / kTileN) * ((M + kRedRows - 1) / kRedRows);
+        cfg.gridDim = dim3((unsigned)red_grid);
+        cfg.blockDim = dim3(kRedThreads);
+        cfg.dynamicSmemBytes = 0;
+        e = red_grid <= 2 * l->grid ? cudaLaunchKernelEx(&cfg, linear_reduce_kernel<8>, p)
+                                    : cudaLaunchKernelEx(&cfg, linear_reduce_kernel<4>, p);
+    }
     if (e != cudaSuccess) return err(ISV_ECUDA, "isv_linear_forward: %s", cudaGetErrorString(e));
     return ISV_OK;
 }
@@ -567,7 +597,6 @@ int isv_linear_status(isv_linear *l, uint32_t *status_out) {
     if (e != cudaSuccess) return err(ISV_ECUDA, "isv_linear_status: %s", cudaGetErrorString(e));
     if (*status_out) {
         cudaMemset(l->status, 0, 4);
-        cudaMemset(l->tickets, 0, (size_t)(l->N / kTileN) * 4);
         return err(ISV_EDEVICE_STATUS, "the linear kernel reported status 0x%x", *status_out);
     }
     return ISV_OK;

@@ -33,7 +33,7 @@ def test_linear_matches_reference(M, N, K, dtype):
     torch.cuda.synchronize()
     l = B.isv_linear_create(wd, N, K, B.ISV_F16 if dtype == "f16" else B.ISV_BF16, max(M, 16), stream.cuda_stream)
     try:
-        for rep in range(2):                         # the second call meets the first one's scratch and tickets
+        for rep in range(2):                         # the second call meets the first one's scratch
             B.isv_linear_forward(l, xd, y16, y32, M)
             assert B.isv_linear_status(l) == 0
             ref = ol.linear(values(x, dtype), values(w, dtype))
