@@ -585,18 +585,19 @@ def point_summary(p):
 LINEAR_MODELS = {"llama7b": (4096, 11008, True), "opt2.7b": (2560, 10240, False)}
 
 
-def linear_layers_bench(cx: Ctx, model="llama7b", batches=(1, 32, 128), iters=40):
+def linear_layers_bench(cx: Ctx, model="llama7b", batches=(1, 32, 128), iters=40, eager=False):
     """Times the four projections of one transformer layer (fused QKV, output, MLP up, MLP down) through
     isv_linear_forward: the linear-layer term of T_compute^d.  Each call streams its weight matrix once;
     the figure of merit is weight bytes / time against the HBM rate.  Several weight buffers are cycled so
     that no call finds its weights in L2, and the calls are captured in a CUDA graph so that the host's
-    launch rate does not enter."""
+    launch rate does not enter (`eager`: plain calls instead, so that a profiler sees ordinary launches)."""
     import torch
     from paper_2504_11816_b200 import binding as B
     h1, h2, gated = LINEAR_MODELS[model]
     shapes = [("qkv", 3 * h1, h1), ("out", h1, h1), ("mlp_up", (2 if gated else 1) * h2, h1), ("mlp_down", h1, h2)]
     stream = torch.cuda.Stream()
-    res = {"model": model, "hbm_peak_GBps": cx.hbm_gbs, "timed": "CUDA graph of the calls", "batches": []}
+    res = {"model": model, "hbm_peak_GBps": cx.hbm_gbs, "timed": "plain calls" if eager else "CUDA graph of the calls",
+           "batches": []}
     floor_us = sum(N * K * 2 for _, N, K in shapes) / (cx.hbm_gbs * 1e9) * 1e6
     for M in batches:
         rows, total_s = [], 0.0
@@ -616,16 +617,20 @@ def linear_layers_bench(cx: Ctx, model="llama7b", batches=(1, 32, 128), iters=40
                     B.isv_linear_forward(hl, x, y, None, M)
                 assert B.isv_linear_status(hs[0]) == 0
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(graph, stream=stream):
+                def calls():
                     for i in range(iters):
                         B.isv_linear_forward(hs[i % copies], x, y, None, M)
-                graph.replay()
+                graph = None
+                if not eager:
+                    graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(graph, stream=stream):
+                        calls()
+                    graph.replay()
                 stream.synchronize()
                 torch.cuda.synchronize()
                 with torch.cuda.stream(stream):
                     e0.record(stream)
-                    graph.replay()
+                    calls() if eager else graph.replay()
                     e1.record(stream)
                 stream.synchronize()
                 torch.cuda.synchronize()
@@ -644,6 +649,19 @@ def linear_layers_bench(cx: Ctx, model="llama7b", batches=(1, 32, 128), iters=40
         res["batches"].append({"batch": M, "rows": rows, "us_per_layer": total_s * 1e6,
                                "floor_us_per_layer": floor_us, "frac": floor_us / (total_s * 1e6)})
     return res
+
+
+def run_linear(args):
+    """`--workload linear`: the decode linear layers alone, at one batch size (`--batch`, default 32) and
+    `--steps` calls per matrix; its own JSON line, not the metric's."""
+    cx = Ctx(args)
+    from paper_2504_11816_b200 import binding as B
+    B.lib()
+    res = linear_layers_bench(cx, batches=(args.batch or 32,), iters=args.steps, eager=args.linear_eager)
+    if cx.rank == 0:
+        print(json.dumps({"linear_layers": res}))
+    if cx.world > 1:
+        cx.dist.destroy_process_group()
 
 
 # ---------------------------------------------------------------- our arm: the line
@@ -770,6 +788,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-linear", action="store_true", help="skip the decode linear layers' figures")
+    ap.add_argument("--linear-eager", action="store_true",
+                    help="with --workload linear: plain calls instead of a CUDA graph (for a profiler)")
     ap.add_argument("--selftest-launch", action="store_true",
                     help="exercise the launcher and the rank reductions on CPU (gloo); no GPU work")
     args = ap.parse_args()
@@ -783,6 +803,9 @@ def main():
                 raise SystemExit(f"--gpus {args.gpus} but only {torch.cuda.device_count()} GPUs are visible")
         raise SystemExit(spawn_ranks(args.gpus))
     from paper_2504_11816_b200 import workloads as W
+    if args.workload == "linear" and args.impl == "ours" and not args.selftest_launch:
+        args.steps = args.steps or 40
+        return run_linear(args)
     if args.workload != "sweep" and args.workload not in W.CONFIGS:
         raise SystemExit(f"unknown workload {args.workload!r}")
     if args.selftest_launch:

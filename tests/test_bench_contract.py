@@ -93,3 +93,14 @@ def test_default_run_is_the_offload_sweep():
     assert d["min_frac_over_sweep"] == min(p["combined_roofline_frac"] for p in d["sweep"])
     assert d["steps"] == 3 and d["warmup"] == 3 and d["e2e"]["value"] > 0
     assert d["linear_layers"]["batches"][0]["rows"][0]["weight_GBps"] > 0
+
+
+@pytest.mark.gpu
+def test_linear_workload_times_the_four_projections_alone():
+    """`--workload linear`: the decode linear layers by themselves, as plain calls (the form a profiler is given)."""
+    d = _run("--workload", "linear", "--batch", "8", "--steps", "4", "--linear-eager")
+    (b,) = d["linear_layers"]["batches"]
+    assert b["batch"] == 8 and [r["layer"] for r in b["rows"]] == ["qkv", "out", "mlp_up", "mlp_down"]
+    for r in b["rows"]:
+        assert r["weight_GBps"] > 0 and r["max_abs_diff_vs_fp32_gemm"] < 0.05
+    assert d["linear_layers"]["timed"] == "plain calls" and 0 < b["frac"] < 1.2
