@@ -47,7 +47,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if p.wait() != 0:
             raise RuntimeError("nvcc failed: " + " ".join(cmd))
     if force or procs or _stale(LIB, objs):
-        cmd = [_nvcc(), "-shared", "-o", LIB] + objs
+        cmd = [_nvcc(), "-shared"] + NVCC_FLAGS[:2] + ["-o", LIB] + objs
         subprocess.run(cmd, check=True)
     return LIB
 
