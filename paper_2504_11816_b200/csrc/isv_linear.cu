@@ -145,17 +145,26 @@ struct LinearParams {
     int32_t grid_main;       // CTAs of linear_kernel (the reduction needs the same cut)
 };
 
-__device__ __forceinline__ void store_out(const LinearParams &p, int m, int n, float v) {
-    const size_t idx = (size_t)m * p.N + n;
-    if (p.y_f32) p.y_f32[idx] = v;
-    if (p.y) {
-        uint16_t *o = reinterpret_cast<uint16_t *>(p.y) + idx;
-        if (p.bf16) {
-            const __nv_bfloat16 h = __float2bfloat16_rn(v);
-            *o = *reinterpret_cast<const uint16_t *>(&h);
-        } else {
-            const __half h = __float2half_rn(v);
-            *o = *reinterpret_cast<const uint16_t *>(&h);
+// One epilogue thread's 16 accumulator values (tokens c0 .. c0 + 15 of one weight row) to memory: as fp32
+// at f32[token * f32_stride] (F32), as 16-bit values at h16[token * h16_stride] (H16), tokens beyond M left out.
+// The destinations are chosen once per segment, outside the loop over the tokens.
+template <bool F32, bool H16, bool BF16>
+__device__ __forceinline__ void put16(const uint32_t (&r)[16], int c0, int M, float *f32, size_t f32_stride,
+                                      uint16_t *h16, size_t h16_stride) {
+    const bool whole = c0 + 16 <= M;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        if (!whole && c0 + j >= M) break;
+        const float v = __uint_as_float(r[j]);
+        if (F32) f32[(size_t)(c0 + j) * f32_stride] = v;
+        if (H16) {
+            if (BF16) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(v);
+                h16[(size_t)(c0 + j) * h16_stride] = *reinterpret_cast<const uint16_t *>(&h);
+            } else {
+                const __half h = __float2half_rn(v);
+                h16[(size_t)(c0 + j) * h16_stride] = *reinterpret_cast<const uint16_t *>(&h);
+            }
         }
     }
 }
@@ -345,18 +354,21 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             }
             float *slot = p.partials + (size_t)(2 * cta + (first_seg ? 0 : 1)) * p.M * kTileN;
             const int n = t * kTileN + row;
+            // a partial goes to the CTA's slot as fp32 rows of 128; a whole tile straight to the outputs
+            float *f32 = complete ? (p.y_f32 ? p.y_f32 + n : nullptr) : slot + row;
+            uint16_t *h16 = complete && p.y ? reinterpret_cast<uint16_t *>(p.y) + n : nullptr;
+            const size_t f32_stride = complete ? (size_t)p.N : (size_t)kTileN;
+            const int mode = (f32 ? 1 : 0) | (h16 ? (p.bf16 ? 4 : 2) : 0);
             for (int c0 = 0; c0 < p.mma_n; c0 += 16) {
                 uint32_t r[16];
                 tmem_ld_32x32b_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(b * p.mma_n + c0), r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int m = c0 + j;
-                    if (m < p.M) {
-                        const float v = __uint_as_float(r[j]);
-                        if (complete) store_out(p, m, n, v);
-                        else slot[(size_t)m * kTileN + row] = v;
-                    }
+                switch (mode) {
+                case 1: put16<true, false, false>(r, c0, p.M, f32, f32_stride, h16, (size_t)p.N); break;
+                case 2: put16<false, true, false>(r, c0, p.M, f32, f32_stride, h16, (size_t)p.N); break;
+                case 3: put16<true, true, false>(r, c0, p.M, f32, f32_stride, h16, (size_t)p.N); break;
+                case 4: put16<false, true, true>(r, c0, p.M, f32, f32_stride, h16, (size_t)p.N); break;
+                default: put16<true, true, true>(r, c0, p.M, f32, f32_stride, h16, (size_t)p.N); break;
                 }
             }
             // the accumulator may be overwritten by the segment after next
