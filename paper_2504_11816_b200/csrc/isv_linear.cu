@@ -39,8 +39,11 @@ namespace {
 
 constexpr int kTileN = 128;        // weight rows per CTA (MMA M)
 constexpr int kSwzK = 64;          // elements of one 128-byte swizzle row
-constexpr int kSub = 2;            // swizzle rows (sub-tiles along K) per ring stage, fetched by one TMA copy
-constexpr int kTileK = kSwzK * kSub;   // elements per ring stage along K
+// A ring stage holds KS sub-tiles along K (KS swizzle rows of 64 elements per matrix row), fetched by one TMA
+// copy per operand: KS = 4 (512 contiguous bytes of every weight row per copy) where two such stages fit beside
+// the activation tiles, else KS = 2.  Measured on B200: 4 is 1-2 % faster than 2 up to 32 tokens, 1 is slower.
+constexpr int kMinTileK = 2 * kSwzK;   // K must be a multiple of this
+constexpr int kWideMaxTokens = 32;     // padded batch up to which KS = 4 is chosen
 constexpr int kMmaK = 16;          // K of one tcgen05.mma for 16-bit operands
 constexpr int kThreads = 192;      // warp 0: TMA, warp 1: MMA + tensor memory, warps 2-5: epilogue
 constexpr uint32_t kSpin = 1u << 22;
@@ -78,7 +81,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return false;
 }
 // 3-D tiled TMA load.  The matrices are described as [K / 64][rows][64 elements], so that one box of
-// {64, rows, kSub} lands as kSub consecutive [rows][64] sub-tiles, each in the 128-byte swizzle.
+// {64, rows, KS} lands as KS consecutive [rows][64] sub-tiles, each in the 128-byte swizzle.
 // x = 0 always (a multiple of 8 elements, as the 16-byte rule for the innermost coordinate asks).
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int row, int kchunk, uint32_t bar) {
     asm volatile(
@@ -142,6 +145,7 @@ struct LinearParams {
     int32_t M, N, K;
     int32_t mma_n;           // batch padded to a multiple of 16
     int32_t stages, tmem_cols, bf16;
+    int32_t tile_k;          // elements per ring stage along K (64 * KS)
     int32_t grid_main;       // CTAs of linear_kernel (the reduction needs the same cut)
 };
 
@@ -203,18 +207,20 @@ struct Cut {
     __device__ int range_of(long long x) const { return (int)(((x + 1) * n - 1) / total); }
     __device__ static Cut of(const LinearParams &p, int grid) {
         Cut c;
-        c.total = (long long)(p.N / kTileN) * (p.K / kTileK);
+        c.total = (long long)(p.N / kTileN) * (p.K / p.tile_k);
         c.n = (int)min((long long)grid, c.total);
         return c;
     }
 };
 
+template <int KS>
 __global__ void __launch_bounds__(kThreads, 2)
 linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const LinearParams p) {
     extern __shared__ uint8_t smem_raw[];
     // the 128-byte swizzle wants tile bases on 1024-byte boundaries of the shared address space
     uint8_t *smem = smem_raw + ((1024u - (s32(smem_raw) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kTileK = kSwzK * KS;
     const int kblocks = p.K / kTileK;
     const Cut cut = Cut::of(p, gridDim.x);
     const int cta = blockIdx.x;
@@ -260,7 +266,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             const uint32_t bar = s32(&full[it]);
             mbar_expect_tx(bar, a_bytes + b_bytes);
             tma_load_3d(s32(ring + (size_t)it * stage_bytes), &map_w, (int)(f / kblocks) * kTileN,
-                        (int)(f % kblocks) * kSub, bar);
+                        (int)(f % kblocks) * KS, bar);
         }
     }
     if (warp == 1) {   // tensor memory: two accumulators of mma_n columns, power-of-two total
@@ -280,7 +286,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
             asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int it = 0; it < prefill; ++it)
                 tma_load_3d(s32(ring + (size_t)it * stage_bytes + a_bytes), &map_x, 0,
-                            (int)((f0 + it) % kblocks) * kSub, s32(&full[it]));
+                            (int)((f0 + it) % kblocks) * KS, s32(&full[it]));
             int it = prefill;
             for (long long f = f0 + prefill; f < f1; ++f, ++it) {
                 const int t = (int)(f / kblocks), kb = (int)(f % kblocks);
@@ -290,8 +296,8 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                 const uint32_t bar = s32(&full[s]);
                 uint8_t *st = ring + (size_t)s * stage_bytes;
                 mbar_expect_tx(bar, a_bytes + b_bytes);
-                tma_load_3d(s32(st), &map_w, t * kTileN, kb * kSub, bar);
-                tma_load_3d(s32(st + a_bytes), &map_x, 0, kb * kSub, bar);
+                tma_load_3d(s32(st), &map_w, t * kTileN, kb * KS, bar);
+                tma_load_3d(s32(st + a_bytes), &map_x, 0, kb * KS, bar);
             }
         }
     } else if (warp == 1) {
@@ -313,7 +319,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = s32(ring + (size_t)s * stage_bytes);
 #pragma unroll
-                    for (int sub = 0; sub < kSub; ++sub) {
+                    for (int sub = 0; sub < KS; ++sub) {
                         const uint64_t da = smem_desc_sw128(a_addr + sub * (kTileN * kSwzK * 2));
                         const uint64_t db = smem_desc_sw128(a_addr + a_bytes + sub * (p.mma_n * kSwzK * 2));
 #pragma unroll
@@ -409,7 +415,7 @@ __device__ __forceinline__ float4 ldcg_if(const float *src, bool pred) {
 
 template <int kFly>
 __global__ void __launch_bounds__(kRedThreads, kFly == 4 ? 4 : 2) linear_reduce_kernel(const LinearParams p) {
-    const int kblocks = p.K / kTileK;
+    const int kblocks = p.K / p.tile_k;
     const Cut cut = Cut::of(p, p.grid_main);
     const int groups = (p.M + kRedRows - 1) / kRedRows;
     const int t = blockIdx.x / groups, m0 = (blockIdx.x % groups) * kRedRows;
@@ -466,14 +472,14 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// Map of a row-major [rows][K] 16-bit matrix seen as [K / 64][rows][64], boxes of kSub x box_rows x 64
+// Map of a row-major [rows][K] 16-bit matrix seen as [K / 64][rows][64], boxes of ks x box_rows x 64
 // elements, 128-byte swizzle, zero fill outside the matrix.
-int make_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows, bool bf16) {
+int make_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows, int ks, bool bf16) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return err(ISV_ECUDA, "cuTensorMapEncodeTiled is not available from this driver");
     const cuuint64_t dims[3] = {(cuuint64_t)kSwzK, (cuuint64_t)rows, (cuuint64_t)(K / kSwzK)};
     const cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)kSwzK * 2};   // bytes: next row, next 64-element chunk
-    const cuuint32_t box[3] = {(cuuint32_t)kSwzK, (cuuint32_t)box_rows, (cuuint32_t)kSub};
+    const cuuint32_t box[3] = {(cuuint32_t)kSwzK, (cuuint32_t)box_rows, (cuuint32_t)ks};
     const cuuint32_t estr[3] = {1, 1, 1};
     const CUresult r = fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
                           const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -490,10 +496,11 @@ struct isv_linear {
     int N = 0, K = 0, max_M = 0;
     bool bf16 = false;
     cudaStream_t stream = nullptr;
-    CUtensorMap map_w;
+    CUtensorMap map_w[2];   // stages of 2 and of 4 sub-tiles along K
+    bool has_ks[2] = {false, false};
     int grid = 1;
     float *partials = nullptr;
-    bool split = false;   // some tile is shared by several CTAs: the reduction kernel follows every launch
+    bool split[2] = {false, false};   // some tile is shared by several CTAs: the reduction kernel follows every launch
     uint32_t *status = nullptr;
     int smem_optin = 0;
 };
@@ -515,7 +522,7 @@ int isv_linear_create(isv_linear **out, const void *w_dev, int32_t N, int32_t K,
     *out = nullptr;
     if (!w_dev || (reinterpret_cast<uintptr_t>(w_dev) & 15u)) return err(ISV_EINVAL, "w must be non-null, 16-byte aligned");
     if (N < kTileN || N % kTileN != 0) return err(ISV_EINVAL, "N (%d) must be a positive multiple of %d", N, kTileN);
-    if (K < kTileK || K % kTileK != 0) return err(ISV_EINVAL, "K (%d) must be a positive multiple of %d", K, kTileK);
+    if (K < kMinTileK || K % kMinTileK != 0) return err(ISV_EINVAL, "K (%d) must be a positive multiple of %d", K, kMinTileK);
     if (max_M < 1 || max_M > 256) return err(ISV_EINVAL, "max_M (%d) must be in [1, 256]", max_M);
     if (dtype != ISV_F16 && dtype != ISV_BF16) return err(ISV_EINVAL, "dtype must be ISV_F16 or ISV_BF16");
     isv_linear *l = new (std::nothrow) isv_linear();
@@ -529,19 +536,25 @@ int isv_linear_create(isv_linear **out, const void *w_dev, int32_t N, int32_t K,
     if (e != cudaSuccess) { delete l; return err(ISV_ECUDA, "isv_linear_create: %s", cudaGetErrorString(e)); }
     const int n_tiles = N / kTileN;
     l->grid = sms;                      // persistent: one CTA per SM (two per SM with half the ring each measured no faster)
-    int rc = make_map(&l->map_w, w_dev, N, K, kTileN, l->bf16);
-    if (rc) { delete l; return rc; }
-    {   // the kernel's cut of the (tile, K block) list: a range border inside a tile splits that tile
-        const long long kblocks = K / kTileK, total = (long long)n_tiles * kblocks;
+    for (int v = 0; v < 2; ++v) {       // variant v: stages of KS = 2 << v sub-tiles
+        const int ks = 2 << v;
+        if (K % (kSwzK * ks) != 0) continue;
+        l->has_ks[v] = true;
+        int rc = make_map(&l->map_w[v], w_dev, N, K, kTileN, ks, l->bf16);
+        if (rc) { delete l; return rc; }
+        // the kernel's cut of the (tile, K block) list: a range border inside a tile splits that tile
+        const long long kblocks = K / (kSwzK * ks), total = (long long)n_tiles * kblocks;
         const long long n = std::min<long long>(l->grid, total);
-        for (long long c = 1; c < n && !l->split; ++c) l->split = (total * c / n) % kblocks != 0;
+        for (long long c = 1; c < n && !l->split[v]; ++c) l->split[v] = (total * c / n) % kblocks != 0;
     }
     e = cudaMalloc((void **)&l->status, 4);
     if (e == cudaSuccess) e = cudaMemset(l->status, 0, 4);
     if (e == cudaSuccess) e = cudaMalloc((void **)&l->partials, (size_t)2 * l->grid * max_M * kTileN * 4);
     // the kernel also has a few bytes of static shared memory: leave room for them under the limit
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, l->smem_optin - 1024);
+        e = cudaFuncSetAttribute(linear_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, l->smem_optin - 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(linear_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, l->smem_optin - 1024);
     if (e != cudaSuccess) {
         cudaGetLastError();
         isv_linear_free(l);
@@ -565,19 +578,32 @@ int isv_linear_forward(isv_linear *l, const void *x_dev, void *y_dev, float *y_f
     int cols = 32;
     while (cols < 2 * p.mma_n) cols *= 2;        // two accumulators
     p.tmem_cols = cols;
-    const size_t a_bytes = (size_t)kTileN * kTileK * 2, b_bytes = (size_t)p.mma_n * kTileK * 2;
-    const size_t stage_bytes = a_bytes + ((b_bytes + 1023) & ~(size_t)1023);
     const size_t fixed = 1024 /* alignment slack */ + 1024 /* static */ + 512 /* barriers, slots */;
     // about 200 KB of ring (measured on B200: 100 -> 180 KB is 8-10 % faster on the large projections although
-    // the next launch's CTA then no longer fits beside this one's to prefetch its weights early)
+    // the next launch's CTA then no longer fits beside this one's to prefetch its weights early); 216 KB where
+    // that is what two or three of the wider stages take
     size_t ring_budget = 200u << 10;
     if (const char *e = getenv("ISV_LINEAR_RING_KB")) ring_budget = (size_t)std::max(32, std::min(220, atoi(e))) << 10;   // tuning knob
-    int stages = (int)std::min<size_t>(std::max<size_t>(2, ring_budget / stage_bytes), ((size_t)l->smem_optin - fixed) / stage_bytes);
+    int v = 0, stages = 0;                        // stage variant: KS = 2 << v
+    size_t stage_bytes = 0;
+    // ISV_LINEAR_KS (tuning knob) = 2 or 4 asks for that stage width where the matrix and the batch allow it
+    const int asked = getenv("ISV_LINEAR_KS") ? atoi(getenv("ISV_LINEAR_KS")) : 0;
+    for (int pass = asked ? 0 : 1; pass < 2 && stages < 2; ++pass)
+        for (int cand = 1; cand >= 0 && stages < 2; --cand) {
+            if (!l->has_ks[cand]) continue;
+            if (pass == 0 ? asked != (2 << cand) : (cand == 1 && p.mma_n > kWideMaxTokens)) continue;
+            const size_t tile_k = (size_t)kSwzK * (2 << cand);
+            const size_t sb = (size_t)kTileN * tile_k * 2 + (((size_t)p.mma_n * tile_k * 2 + 1023) & ~(size_t)1023);
+            const size_t budget = (cand == 1 && !getenv("ISV_LINEAR_RING_KB")) ? (216u << 10) : ring_budget;
+            const int st = (int)std::min<size_t>(std::max<size_t>(2, budget / sb), ((size_t)l->smem_optin - fixed) / sb);
+            if (st >= 2) { v = cand; stage_bytes = sb; stages = st; }
+        }
     if (stages < 2) return err(ISV_EINVAL, "shared memory too small for this batch");
     p.stages = stages;
+    p.tile_k = kSwzK * (2 << v);
     const size_t smem = 1024 + (size_t)stages * stage_bytes + (2 * stages + 4) * 8 + 64;
     CUtensorMap map_x;
-    int rc = make_map(&map_x, x_dev, M, l->K, p.mma_n, l->bf16);   // rows beyond M read as zeros
+    int rc = make_map(&map_x, x_dev, M, l->K, p.mma_n, 2 << v, l->bf16);   // rows beyond M read as zeros
     if (rc) return rc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(l->grid);
@@ -589,8 +615,9 @@ int isv_linear_forward(isv_linear *l, const void *x_dev, void *y_dev, float *y_f
     attr[0].val.programmaticStreamSerializationAllowed = 1;   // see the kernel's griddepcontrol use
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_kernel, l->map_w, map_x, p);
-    if (e == cudaSuccess && l->split) {
+    cudaError_t e = v == 1 ? cudaLaunchKernelEx(&cfg, linear_kernel<4>, l->map_w[1], map_x, p)
+                           : cudaLaunchKernelEx(&cfg, linear_kernel<2>, l->map_w[0], map_x, p);
+    if (e == cudaSuccess && l->split[v]) {
         const int red_grid = (l->N / kTileN) * ((M + kRedRows - 1) / kRedRows);
         cfg.gridDim = dim3((unsigned)red_grid);
         cfg.blockDim = dim3(kRedThreads);

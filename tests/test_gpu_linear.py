@@ -23,6 +23,8 @@ def _case(M, N, K, dtype, seed):
 @pytest.mark.parametrize("M,N,K,dtype", [
     (1, 128, 128, "f16"), (5, 256, 512, "f16"), (16, 128, 1024, "bf16"), (32, 512, 4096, "f16"),
     (33, 384, 2048, "bf16"), (100, 256, 1024, "f16"), (256, 256, 512, "f16"), (64, 1408, 1024, "bf16"),
+    # every CTA walks more K blocks than its ring holds: wide stages (few tokens) and narrow ones (many)
+    (8, 4096, 8192, "f16"), (128, 2048, 4096, "bf16"),
 ])
 def test_linear_matches_reference(M, N, K, dtype):
     x, w = _case(M, N, K, dtype, seed=M * 7 + N)
