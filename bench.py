@@ -585,7 +585,7 @@ def point_summary(p):
 LINEAR_MODELS = {"llama7b": (4096, 11008, True), "opt2.7b": (2560, 10240, False)}
 
 
-def linear_layers_bench(cx: Ctx, model="llama7b", batches=(1, 32, 128), iters=40, eager=False):
+def linear_layers_bench(cx: Ctx, model="llama7b", batches=(1, 32, 64, 128), iters=40, eager=False):
     """Times the four projections of one transformer layer (fused QKV, output, MLP up, MLP down) through
     isv_linear_forward: the linear-layer term of T_compute^d.  Each call streams its weight matrix once;
     the figure of merit is weight bytes / time against the HBM rate.  Several weight buffers are cycled so
