@@ -91,7 +91,7 @@ typedef struct {
     int32_t  max_tokens_per_seq; /* capacity per sequence (L_in + L_out)                        */
     uint64_t perm_seed;          /* 0 = physical block ids handed out in order; otherwise they  */
                                  /* follow a seeded permutation (host pool ids stay compact)    */
-    uint64_t chunk_bytes;        /* staging chunk size; 0 = 1/8 of a layer's host pool in [32, 128] MiB */
+    uint64_t chunk_bytes;        /* staging chunk size; 0 = 128 MiB or a layer's host pool if smaller */
     int32_t  ring_depth;         /* staging ring buffers; 0 = 3                                 */
     int32_t  max_ctas;           /* cap on the resident kernel's grid; 0 = one CTA per SM.      */
                                  /* The KV blocks are cut evenly over the grid's warps, so this */

@@ -302,12 +302,12 @@ inline const char *make_geometry(const isv_kv_desc &d, Geometry *out) {
     if (d.max_ctas < 0) return "max_ctas must be >= 0";
     g.max_ctas = d.max_ctas;
     if ((long long)g.max_seqs * g.NB * g.Hkv * g.P >= (1ll << 31)) return "max_seqs * blocks * heads too large";
-    // default chunk: an eighth of a layer's host pool, within [32 MiB, 128 MiB] (measured on B200 at the 13B shape:
-    // 128 MiB chunks reach 0.995 of the probed link rate where 32 MiB chunks reach 0.988-0.992; a small pool
-    // keeps several chunks per layer so that copies and attention still overlap inside a layer)
-    const uint64_t pool_eighth = (uint64_t)g.host_cap * g.block_bytes / 8;
-    g.chunk_bytes = d.chunk_bytes != 0 ? d.chunk_bytes
-                                       : std::min<uint64_t>(128ull << 20, std::max<uint64_t>(32ull << 20, pool_eighth));
+    // default chunk: 128 MiB, or a layer's whole host pool where that is smaller (measured on B200: every copy
+    // costs a few us of link idle time; 128 MiB chunks reach 0.994-0.996 of the probed link rate at the 13B and
+    // OPT-2.7B shapes where 32 MiB chunks reach 0.988-0.992; copies of the next layer run ahead, so even one chunk
+    // per layer keeps the link busy)
+    const uint64_t pool_bytes = std::max<uint64_t>(g.block_bytes, (uint64_t)g.host_cap * g.block_bytes);
+    g.chunk_bytes = d.chunk_bytes != 0 ? d.chunk_bytes : std::min<uint64_t>(128ull << 20, pool_bytes);
     g.chunk_blocks = (int)std::max<uint64_t>(1, g.chunk_bytes / g.block_bytes);
     g.chunk_bytes = (uint64_t)g.chunk_blocks * g.block_bytes;
     g.ring = d.ring_depth == 0 ? 3 : d.ring_depth;
